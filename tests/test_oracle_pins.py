@@ -1,0 +1,462 @@
+"""Pins for the CPU oracle: every check compares it with something other than itself --
+facts the paper states, closed forms, textbook bounds, library routines (numpy / scipy /
+torch in fp64) in the special cases that reduce to them, and brute force on tiny inputs."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import scipy.special
+import torch
+
+import oracle
+from oracle import Table
+import nm_inputs
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def paper_facts():
+    facts = {}
+    with open(os.path.join(HERE, "golden", "paper_facts.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split("=")
+                facts[k.strip()] = float(v)
+    return facts
+
+
+def np_f(func):
+    return {
+        oracle.GELU: lambda x: 0.5 * x * (1 + scipy.special.erf(x / np.sqrt(2.0))),
+        oracle.EXP: np.exp,
+        oracle.RECIP: lambda x: 1.0 / x,
+        oracle.RSQRT: lambda x: 1.0 / np.sqrt(x),
+        oracle.RELU: lambda x: np.maximum(x, 0.0),
+        oracle.SQRT: np.sqrt,
+        oracle.IDENTITY: lambda x: x,
+    }[func]
+
+
+def np_f2max(func, lo, hi):
+    """max |f''| on [lo, hi] from a dense numerical second difference (independent of the oracle)."""
+    x = np.linspace(lo, hi, 200001)
+    f = np_f(func)(x)
+    h = x[1] - x[0]
+    return np.max(np.abs(f[2:] - 2 * f[1:-1] + f[:-2])) / h ** 2
+
+
+RANGES = {oracle.GELU: (-4.0, 4.0), oracle.EXP: (-8.0, 0.0), oracle.RECIP: (8.0, 128.0),
+          oracle.RSQRT: (0.25, 4.0), oracle.SQRT: (0.25, 4.0)}
+
+
+# ---------------------------------------------------------------- tables ---------
+
+@pytest.mark.parametrize("func", list(RANGES))
+@pytest.mark.parametrize("n", [7, 16, 64, 256])
+def test_table_interpolates_and_is_continuous(func, n):
+    """Section 3.2.1: the end of one segment is the start of the next, so at every breakpoint both
+    neighbouring lines give f(x_i)."""
+    lo, hi = RANGES[func]
+    t = Table.secant(func, n, lo, hi)
+    xs = lo + (hi - lo) * np.arange(n + 1) / n
+    f = np_f(func)(xs)
+    k = t.k.astype(np.float64)
+    b = t.b.astype(np.float64)
+    left = k * xs[:-1] + b       # segment i at its start
+    right = k * xs[1:] + b       # segment i at its end
+    scale = np.maximum(np.abs(f).max(), 1.0)
+    # k, b are stored in fp32: interpolation holds to fp32 rounding of k*x and b
+    tol = 4e-7 * (np.abs(k) * np.abs(xs[:-1]) + np.abs(b) + scale).max()
+    assert np.abs(left - f[:-1]).max() <= tol
+    assert np.abs(right - f[1:]).max() <= tol
+    assert np.abs(right[:-1] - left[1:]).max() <= 2 * tol
+
+
+@pytest.mark.parametrize("func", list(RANGES))
+def test_table_error_bound_shrinks_16x(func):
+    """Linear interpolation error is at most h^2/8 * max|f''|; four times the segments, a
+    sixteenth of the error."""
+    lo, hi = RANGES[func]
+    f2 = np_f2max(func, lo, hi)
+    x = np.linspace(lo, hi, 40001)
+    errs = []
+    for n in (16, 64, 256):
+        t = Table.secant(func, n, lo, hi)
+        y = t(x)
+        err = np.abs(y - np_f(func)(x)).max()
+        h = (hi - lo) / n
+        assert err <= h * h / 8 * f2 * 1.02 + 1e-6
+        errs.append(err)
+    # the 16x law is asymptotic (h small against the curvature scale): strict at 64 -> 256
+    assert 6 < errs[0] / errs[1] < 20
+    assert 12 < errs[1] / errs[2] < 20
+
+
+def test_relu_two_segments_exact():
+    """Section 3: ReLU is already piecewise linear -- two segments reproduce it exactly, in and
+    out of range."""
+    t = Table.secant(oracle.RELU, 2, -6.0, 6.0)
+    assert t.k.tolist() == [0.0, 1.0] and t.b.tolist() == [0.0, 0.0]
+    x = np.concatenate([np.linspace(-100, 100, 4001), [0.0, -0.0, 6.0, -6.0, 1e30, -1e30]])
+    assert np.array_equal(t(x), np.maximum(x, 0.0))
+
+
+def test_identity_table_is_identity():
+    t = Table.secant(oracle.IDENTITY, 64, -3.0, 5.0)
+    assert np.all(t.k == 1.0) and np.all(np.abs(t.b) < 1e-6)
+
+
+def test_gelu_tails_match_paper_statement():
+    fx = paper_facts()
+    lo, hi = fx["gelu_near_zero_at_or_below"], fx["gelu_near_identity_at_or_above"]
+    x = np.linspace(-8, lo, 101)
+    assert np.abs(oracle.exact(oracle.GELU, x)).max() < 5e-3
+    x = np.linspace(hi, 8, 101)
+    assert np.abs(oracle.exact(oracle.GELU, x) - x).max() < 5e-3
+    # and the erf form itself, against scipy
+    x = np.linspace(-6, 6, 1001)
+    assert np.allclose(oracle.exact(oracle.GELU, x), np_f(oracle.GELU)(x), rtol=0, atol=1e-15)
+
+
+def test_out_of_range_extends_end_lines():
+    """Section 3.2.1: inputs outside the range share k, b with the first / last segment."""
+    t = Table.secant(oracle.EXP, 8, -8.0, 0.0)
+    x = np.array([-20.0, -8.5, 0.5, 3.0])
+    y, idx = oracle.pwl_eval(t, x)
+    assert idx.tolist() == [0, 0, 7, 7]
+    exp = np.array([t.k[0] * x[0] + t.b[0], t.k[0] * x[1] + t.b[0], t.k[7] * x[2] + t.b[7],
+                    t.k[7] * x[3] + t.b[7]], np.float64)
+    assert np.allclose(y, exp, rtol=1e-15)
+    # x exactly at x_max belongs to the last segment
+    assert oracle.pwl_eval(t, np.array([0.0]))[1][0] == 7
+
+
+def test_parameter_budget_order_of_magnitude():
+    """Section 5.2: ~1.6 KB / 3.2 KB of extra parameters; 4 tables x 64 segments x (k,b) fp32 = 2 KB."""
+    fx = paper_facts()
+    ours = 4 * 64 * 2 * 4
+    assert fx["extra_params_roberta_bytes"] / 2 <= ours <= fx["extra_params_resnet50_bytes"] * 2
+
+
+# ---------------------------------------------------------------- index ----------
+
+@pytest.mark.parametrize("func,n", [(oracle.GELU, 64), (oracle.EXP, 16), (oracle.RECIP, 256), (oracle.RSQRT, 37)])
+def test_index_matches_linear_search_away_from_breakpoints(func, n):
+    lo, hi = RANGES[func]
+    t = Table.secant(func, n, lo, hi)
+    bp = lo + (hi - lo) * np.arange(n + 1) / n
+    rng = np.random.default_rng(3)
+    x = rng.uniform(lo - 1, hi + 1, 20000).astype(np.float32)
+    dist = np.abs(x[:, None].astype(np.float64) - bp[None, :]).min(axis=1)
+    x = x[dist > 1e-4 * (hi - lo) / n * 64]
+    _, idx = oracle.pwl_eval(t, x)
+    brute = np.clip(np.searchsorted(bp, x.astype(np.float64), side="right") - 1, 0, n - 1)
+    assert np.array_equal(idx, brute)
+
+
+def test_index_is_one_correctly_rounded_fp32_fma():
+    """The index is floor(fma(x, inv_h, off)) with a single fp32 rounding: checked against exact
+    rational arithmetic."""
+    t = Table.secant(oracle.GELU, 64, -4.0, 4.0)
+    inv_h = np.float32(64 / 8.0)
+    off = np.float32(4.0 * 64 / 8.0)
+    t2 = Table.secant(oracle.RSQRT, 37, 0.25, 4.0)
+    span = float(np.float32(4.0)) - float(np.float32(0.25))
+    inv_h2 = np.float32(37 / span)
+    off2 = np.float32(-0.25 * 37 / span)
+    pts = nm_inputs.pwl_probe_points(-4.0, 4.0, 64, 500, 1)
+    pts = pts[np.isfinite(pts)]
+    for tab, ih, of, n in ((t, inv_h, off, 64), (t2, inv_h2, off2, 37)):
+        for x in pts[:700]:
+            exact_u = Fraction(float(x)) * Fraction(float(ih)) + Fraction(float(of))
+            u = np.float32(exact_u)  # Fraction -> double -> float can double-round; guard below
+            lo_ = np.nextafter(u, np.float32(-np.inf))
+            hi_ = np.nextafter(u, np.float32(np.inf))
+            cands = sorted({float(lo_), float(u), float(hi_)}, key=lambda c: abs(Fraction(c) - exact_u))
+            u = cands[0]
+            # skip exact ties between two floats (none expected for these constants)
+            if len(cands) > 1 and abs(Fraction(cands[0]) - exact_u) == abs(Fraction(cands[1]) - exact_u):
+                continue
+            want = min(max(math.floor(u), 0), n - 1)
+            assert int(tab.index(np.array([x]))[0]) == want
+
+
+def test_index_nan_selects_segment_zero():
+    t = Table.secant(oracle.GELU, 64, -4.0, 4.0)
+    y, idx = oracle.pwl_eval(t, np.array([np.nan]))
+    assert idx[0] == 0 and np.isnan(y[0])
+
+
+def test_f32_eval_is_fma():
+    t = Table.secant(oracle.EXP, 64, -8.0, 0.0)
+    x = nm_inputs.pwl_probe_points(-8.0, 0.0, 64, 300, 5)
+    x = x[np.isfinite(x)]
+    y, idx = oracle.pwl_eval_f32(t, x)
+    for xi, yi, s in zip(x[:400], y[:400], idx[:400]):
+        ex = Fraction(float(t.k[s])) * Fraction(float(xi)) + Fraction(float(t.b[s]))
+        # correctly rounded: no other float is closer
+        for nb in (np.nextafter(yi, np.float32(np.inf)), np.nextafter(yi, np.float32(-np.inf))):
+            assert abs(Fraction(float(yi)) - ex) <= abs(Fraction(float(nb)) - ex)
+
+
+# ---------------------------------------------------------------- linear ---------
+
+def test_linear_brute_force_tiny():
+    rng = np.random.default_rng(0)
+    A = rng.standard_normal((3, 5))
+    W = rng.standard_normal((4, 5))
+    bias = rng.standard_normal(4)
+    res = rng.standard_normal((3, 4))
+    out = oracle.linear(A, W, bias, res)
+    for m in range(3):
+        for j in range(4):
+            s = sum(A[m, c] * W[j, c] for c in range(5)) + bias[j] + res[m, j]
+            assert abs(out[m, j] - s) < 1e-13
+
+
+def test_linear_matches_numpy_and_epilogue_order():
+    """bias -> table -> residual: with the exact 2-segment ReLU table the result must be
+    relu(A W^T + bias) + residual, computed by numpy."""
+    rng = np.random.default_rng(1)
+    A = rng.standard_normal((37, 53))
+    W = rng.standard_normal((29, 53))
+    bias = rng.standard_normal(29)
+    res = rng.standard_normal((37, 29))
+    relu = Table.secant(oracle.RELU, 2, -10.0, 10.0)
+    out, idx = oracle.linear(A, W, bias, res, relu, want_idx=True)
+    pre = A @ W.T + bias
+    assert np.allclose(out, np.maximum(pre, 0) + res, rtol=1e-12, atol=1e-12)
+    assert np.array_equal(idx, (pre.astype(np.float32) >= 0).astype(np.int32))
+    ident = Table.secant(oracle.IDENTITY, 64, -3.0, 3.0)
+    out2 = oracle.linear(A, W, bias, None, ident)
+    assert np.allclose(out2, pre, rtol=1e-6, atol=1e-6)   # b of the identity table is O(1e-7)
+    assert np.allclose(oracle.linear(A, W), A @ W.T, rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- attention ------
+
+def _torch_attention(qkv, B, L, h, d):
+    H = h * d
+    t = torch.from_numpy(qkv).reshape(B, L, 3, h, d)
+    q, k, v = (t[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v)
+    return o.permute(0, 2, 1, 3).reshape(B * L, H).numpy()
+
+
+def test_attention_exact_mode_is_textbook_softmax_attention():
+    B, L, h, d = 2, 24, 3, 8
+    rng = np.random.default_rng(2)
+    qkv = rng.standard_normal((B * L, 3 * h * d))
+    out = oracle.attention(qkv, B, L, h, d, Table.exact(oracle.EXP), Table.exact(oracle.RECIP))
+    assert np.allclose(out, _torch_attention(qkv, B, L, h, d), rtol=1e-10, atol=1e-12)
+
+
+def test_attention_pwl_converges_to_exact_and_uses_final_max():
+    B, L, h, d = 1, 32, 2, 16
+    rng = np.random.default_rng(4)
+    qkv = rng.standard_normal((B * L, 3 * h * d))
+    ref = _torch_attention(qkv, B, L, h, d)
+    errs = []
+    for n in (16, 64, 256):
+        te = Table.secant(oracle.EXP, n, -16.0, 0.0)
+        tr = Table.secant(oracle.RECIP, n, 1.0, float(L))
+        errs.append(np.abs(oracle.attention(qkv, B, L, h, d, te, tr) - ref).max())
+    assert errs[0] > errs[1] > errs[2] and errs[2] < 2e-3
+    # a row whose scores are all equal: e_j = PWLexp(0) for every j, sigma = L * PWLexp(0)
+    q = np.zeros((L, 3 * h * d))
+    q[:, 2 * h * d:] = rng.standard_normal((L, h * d))
+    te = Table.secant(oracle.EXP, 64, -8.0, 0.0)
+    tr = Table.secant(oracle.RECIP, 64, 2.0, 32.0)
+    out = oracle.attention(q, 1, L, h, d, te, tr)
+    e0 = te(np.array([0.0]))[0]
+    r = tr(np.array([L * e0]))[0]
+    want = (e0 * r) * q[:, 2 * h * d:].sum(axis=0, keepdims=True)
+    assert np.allclose(out, np.repeat(want, L, axis=0), rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- layernorm ------
+
+def test_layernorm_exact_mode_is_library_layer_norm():
+    rng = np.random.default_rng(5)
+    z = rng.standard_normal((9, 48)) * 3 + 1
+    g = rng.standard_normal(48)
+    b = rng.standard_normal(48)
+    y = oracle.layernorm(z, g, b, 1e-5, Table.exact(oracle.RSQRT))
+    ref = torch.nn.functional.layer_norm(torch.from_numpy(z), (48,), torch.from_numpy(g), torch.from_numpy(b), 1e-5)
+    assert np.allclose(y, ref.numpy(), rtol=1e-11, atol=1e-12)
+
+
+def test_layernorm_pwl_uses_table_on_variance_plus_eps():
+    rng = np.random.default_rng(6)
+    z = rng.standard_normal((5, 64))
+    t = Table.secant(oracle.RSQRT, 64, 0.25, 4.0)
+    y = oracle.layernorm(z, np.ones(64), np.zeros(64), 1e-5, t)
+    assert np.abs(y.mean(axis=1)).max() < 1e-14
+    v = z.var(axis=1)
+    r = t(v + 1e-5)
+    assert np.allclose(y.std(axis=1), np.sqrt(v) * r, rtol=1e-12)
+
+
+# ---------------------------------------------------------------- encoder layer --
+
+def _torch_encoder_layer(x, w, B, L, h):
+    H = x.shape[1]
+    F = w["W1"].shape[0]
+    layer = torch.nn.TransformerEncoderLayer(H, h, F, dropout=0.0, activation="gelu", batch_first=True,
+                                             norm_first=False, dtype=torch.float64)
+    sd = {
+        "self_attn.in_proj_weight": w["Wqkv"], "self_attn.in_proj_bias": w["bqkv"],
+        "self_attn.out_proj.weight": w["Wo"], "self_attn.out_proj.bias": w["bo"],
+        "linear1.weight": w["W1"], "linear1.bias": w["b1"], "linear2.weight": w["W2"], "linear2.bias": w["b2"],
+        "norm1.weight": w["g1"], "norm1.bias": w["be1"], "norm2.weight": w["g2"], "norm2.bias": w["be2"],
+    }
+    layer.load_state_dict({k: torch.from_numpy(np.asarray(v, np.float64)) for k, v in sd.items()})
+    layer.train(False)
+    with torch.no_grad():
+        torch.backends.mha.set_fastpath_enabled(False)
+        y = layer(torch.from_numpy(np.asarray(x, np.float64)).reshape(B, L, H))
+    return y.reshape(B * L, H).numpy()
+
+
+def _exact_tables():
+    return {"gelu": Table.exact(oracle.GELU), "exp": Table.exact(oracle.EXP),
+            "recip": Table.exact(oracle.RECIP), "rsqrt": Table.exact(oracle.RSQRT)}
+
+
+def _pwl_tables(cfg, n):
+    r = cfg.ranges()
+    return {"gelu": Table.secant(oracle.GELU, n, *r["gelu"]), "exp": Table.secant(oracle.EXP, n, *r["exp"]),
+            "recip": Table.secant(oracle.RECIP, n, *r["recip"]), "rsqrt": Table.secant(oracle.RSQRT, n, *r["rsqrt"])}
+
+
+def test_encoder_layer_exact_mode_is_library_post_ln_layer():
+    cfg = nm_inputs.EncoderConfig("t", "f32", B=2, L=16, H=48, heads=4, F=96)
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=7, random_affine=True)
+    w = {k: v * (5.0 if k.startswith("W") else 1.0) for k, v in layers[0].items()}
+    y = oracle.encoder_layer(x, w, cfg.B, cfg.L, cfg.heads, _exact_tables(), eps=1e-5)
+    ref = _torch_encoder_layer(x, w, cfg.B, cfg.L, cfg.heads)
+    assert np.allclose(y, ref, rtol=1e-9, atol=1e-10)
+
+
+def test_encoder_layer_pwl_approaches_exact_with_more_segments():
+    cfg = nm_inputs.with_(nm_inputs.C1, B=1, L=32, H=64, heads=4, F=128)
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=0)
+    w = {k: v * (4.0 if k.startswith("W") else 1.0) for k, v in layers[0].items()}
+    ref = oracle.encoder_layer(x, w, cfg.B, cfg.L, cfg.heads, _exact_tables())
+    errs = [np.abs(oracle.encoder_layer(x, w, cfg.B, cfg.L, cfg.heads, _pwl_tables(cfg, n)) - ref).max()
+            for n in (16, 64, 256)]
+    assert errs[0] > errs[1] > errs[2]
+    assert errs[2] < 1e-3
+
+
+# ---------------------------------------------------------------- int8 -----------
+
+def test_int8_accumulators_and_epilogue():
+    M, N, K = 19, 23, 96
+    Aq = nm_inputs.int8_matrix((M, K), 1)
+    Wq = nm_inputs.int8_matrix((N, K), 2)
+    rng = np.random.default_rng(3)
+    ws = rng.uniform(1e-4, 3e-4, N).astype(np.float32)
+    bias = (0.1 * rng.standard_normal(N)).astype(np.float32)
+    a_scale = np.float32(0.031)
+    t = Table.secant(oracle.GELU, 64, -4.0, 4.0)
+    r = oracle.linear_i8(Aq, Wq, a_scale, ws, bias, None, t, out_scale=0.05)
+    acc = Aq.astype(np.int64) @ Wq.astype(np.int64).T
+    assert np.array_equal(r["acc"], acc.astype(np.int32))
+    inv = np.float32(1.0) / np.float32(0.05)
+    for m in range(0, M, 3):
+        for j in range(0, N, 2):
+            sc = np.float32(a_scale * ws[j])
+            ex = Fraction(int(acc[m, j])) * Fraction(float(sc)) + Fraction(float(bias[j]))
+            x = np.float32(float(ex))          # |ex| small, 53-bit double then float: check nearest below
+            for nb in (np.nextafter(x, np.float32(np.inf)), np.nextafter(x, np.float32(-np.inf))):
+                if abs(Fraction(float(nb)) - ex) < abs(Fraction(float(x)) - ex):
+                    x = nb
+            s = int(t.index(np.array([x]))[0])
+            assert r["idx"][m, j] == s
+            ey = Fraction(float(t.k[s])) * Fraction(float(x)) + Fraction(float(t.b[s]))
+            y = r["y"][m, j]
+            for nb in (np.nextafter(y, np.float32(np.inf)), np.nextafter(y, np.float32(-np.inf))):
+                assert abs(Fraction(float(y)) - ey) <= abs(Fraction(float(nb)) - ey)
+            q = float(np.clip(np.rint(np.float32(y * inv)), -127, 127))
+            assert r["q"][m, j] == q
+
+
+def test_quantize_round_half_even_and_clamp():
+    x = np.array([0.5, 1.5, 2.5, -0.5, -1.5, 200.0, -200.0, 126.5, 127.4], np.float32)
+    q = oracle.quantize_i8(x, 1.0)
+    assert q.tolist() == [0, 2, 2, 0, -2, 127, -127, 126, 127]
+
+
+# ---------------------------------------------------------------- CNN pieces -----
+
+def test_conv_pool_match_torch():
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((2, 9, 11, 5))
+    W = rng.standard_normal((7, 3, 3, 5))
+    bias = rng.standard_normal(7)
+    for stride, pad in ((1, 1), (2, 1), (2, 0)):
+        out = oracle.conv2d_nhwc(x, W, stride, pad, bias)
+        ref = torch.nn.functional.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2), torch.from_numpy(W).permute(0, 3, 1, 2),
+                                         torch.from_numpy(bias), stride=stride, padding=pad).permute(0, 2, 3, 1).numpy()
+        assert np.allclose(out, ref, rtol=1e-11, atol=1e-11)
+    relu = Table.secant(oracle.RELU, 2, -8.0, 8.0)
+    res = rng.standard_normal((2, 9, 11, 7))
+    out = oracle.conv2d_nhwc(x, W, 1, 1, bias, res, relu)
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2), torch.from_numpy(W).permute(0, 3, 1, 2),
+                                     torch.from_numpy(bias), padding=1).permute(0, 2, 3, 1).numpy()
+    assert np.allclose(out, np.maximum(ref, 0) + res, rtol=1e-11, atol=1e-11)
+    mp = oracle.maxpool_nhwc(x, 3, 2, 1)
+    ref = torch.nn.functional.max_pool2d(torch.from_numpy(x).permute(0, 3, 1, 2), 3, 2, 1).permute(0, 2, 3, 1).numpy()
+    assert np.array_equal(mp, ref)
+    assert np.allclose(oracle.avgpool_nhwc(x), x.mean(axis=(1, 2)), rtol=1e-13)
+
+
+# ---------------------------------------------------------------- Algorithms 2, 3 -
+
+def test_alg2_worked_example_merges_minus2_to_minus1():
+    """Section 3.2.2 / Fig. 3(a): with threshold 0.1 and primary length 0.5 the two primary
+    segments on [-2,-1] of GELU merge into one."""
+    fx = paper_facts()
+    xs = oracle.hsize_startpoints(oracle.GELU, fx["alg2_example_dLx"], fx["alg2_example_dK_th"], -4.0, 4.0)
+    a, b = fx["alg2_example_merged_from"], fx["alg2_example_merged_to"]
+    assert a in xs and b in xs and (a + b) / 2 not in xs
+    assert xs[0] == -4.0 and len(xs) < 16          # fewer than the 16 primary segments
+    # a straight line never opens a new segment; a parabola opens one at every primary step
+    assert len(oracle.hsize_startpoints(oracle.IDENTITY, 0.5, 0.1, -4.0, 4.0)) == 1
+
+
+def test_alg3_bias_correction():
+    """dE is the mean of f minus the mean of the secant; for a convex f it is negative; it removes
+    ~5/6 of the squared error (closed form for small segments), the paper reporting 74-83 %."""
+    fx = paper_facts()
+    paper = {oracle.EXP: fx["alg3_mse_reduction_exp"], oracle.SQRT: fx["alg3_mse_reduction_sqrt"],
+             oracle.RECIP: fx["alg3_mse_reduction_recip"], oracle.GELU: fx["alg3_mse_reduction_gelu"]}
+    for func, (lo, hi) in ((oracle.EXP, (-8.0, 0.0)), (oracle.SQRT, (0.25, 4.0)), (oracle.RECIP, (1.0, 8.0)),
+                           (oracle.GELU, (-4.0, 4.0))):
+        n = 16
+        xs = np.linspace(lo, hi, n + 1)
+        k, b = oracle.secant_points(func, xs)
+        b2, dE = oracle.bias_correct(func, xs, b)
+        x = np.linspace(lo, hi, 160001)[:-1]
+        seg = np.minimum(((x - lo) / (hi - lo) * n).astype(int), n - 1)
+        f = np_f(func)(x)
+        # dE against a numerical mean of (f - secant) per segment
+        num = np.array([(f[seg == i] - (k[i] * x[seg == i] + b[i])).mean() for i in range(n)])
+        assert np.allclose(dE, num, rtol=2e-3, atol=1e-7)
+        if func in (oracle.EXP, oracle.RECIP):
+            assert np.all(dE < 0)
+        if func == oracle.SQRT:
+            assert np.all(dE > 0)
+        mse0 = ((k[seg] * x + b[seg] - f) ** 2).mean()
+        mse1 = ((k[seg] * x + b2[seg] - f) ** 2).mean()
+        red = 100 * (1 - mse1 / mse0)
+        assert 70.0 < red < 84.0
+        assert abs(red - paper[func]) < 12.0
+    # Fig. 3(b): the GELU secant on [-1, 0] is biased (curve below the chord: convex there)
+    k, b = oracle.secant_points(oracle.GELU, np.array([fx["alg3_biased_segment_from"], fx["alg3_biased_segment_to"]]))
+    _, dE = oracle.bias_correct(oracle.GELU, np.array([-1.0, 0.0]), b)
+    assert dE[0] < -0.02
