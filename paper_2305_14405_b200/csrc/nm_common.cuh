@@ -1,0 +1,349 @@
+// Shared device/host pieces of the NeuralMatrix B200 library: the context, the
+// device-resident PWL table and its evaluation primitive, and raw sm_100a PTX
+// wrappers (mbarrier, TMA, tcgen05) with bounded waits.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/nm_b200.h"
+
+// ---------------------------------------------------------------- tables ------
+
+// One PWL table as kernels see it (Section 3.2: k and b pre-stored, indexed by
+// segment number).  kb[s] = (k_s, b_s).
+struct NmTable {
+    int32_t n;
+    float inv_h;  // (float)(n / (x_max - x_min))
+    float off;    // (float)(-x_min * n / (x_max - x_min))
+    float x_min, x_max;
+    int32_t loaded;
+    int32_t pad[2];
+    float2 kb[NM_MAX_SEGMENTS];
+};
+
+struct NmProfRecord {
+    cudaEvent_t start, stop;
+    int kind;
+    double work;
+};
+#define NM_PROF_MAX 8192
+
+struct nm_ctx {
+    int device;
+    NmTable* d_tables;         // NM_NUM_SLOTS tables in device memory
+    NmTable h_tables[NM_NUM_SLOTS];
+    int* d_status;             // device status word (nm_status)
+    int sm_count;
+    int64_t launches;
+    void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
+    int profiling;             // nonzero: bracket every launch with events
+    int prof_count;            // records in use
+    int prof_created;          // event pairs created so far (kept for reuse)
+    NmProfRecord* prof;        // NM_PROF_MAX records, host memory
+};
+
+// Brackets one kernel launch with events when profiling is on; counts the launch always.
+struct NmLaunchScope {
+    nm_ctx* ctx;
+    cudaStream_t st;
+    NmProfRecord* rec;
+    NmLaunchScope(nm_ctx* c, int kind, double work, cudaStream_t s) : ctx(c), st(s), rec(nullptr)
+    {
+        ctx->launches++;
+        if (!ctx->profiling || ctx->prof_count >= NM_PROF_MAX) return;
+        NmProfRecord* r = &ctx->prof[ctx->prof_count];
+        if (ctx->prof_count >= ctx->prof_created) {
+            if (cudaEventCreate(&r->start) != cudaSuccess || cudaEventCreate(&r->stop) != cudaSuccess) return;
+            ctx->prof_created = ctx->prof_count + 1;
+        }
+        r->kind = kind;
+        r->work = work;
+        ctx->prof_count++;
+        rec = r;
+        cudaEventRecord(r->start, st);
+    }
+    ~NmLaunchScope()
+    {
+        if (rec) cudaEventRecord(rec->stop, st);
+    }
+};
+
+// Segment number of x: one fp32 fused multiply-add, floor, clamp to [0, n-1];
+// inputs outside the range land in the end segments (Section 3.2.1), NaN in 0.
+__device__ __forceinline__ int nm_pwl_index(float x, float inv_h, float off, float nm1)
+{
+    float u = __fmaf_rn(x, inv_h, off);
+    u = fminf(fmaxf(u, 0.0f), nm1);
+    return __float2int_rd(u);
+}
+
+// Per-lane replicated table in shared memory: entry s of lane l lives at
+// rep[s * 32 + l], so a warp's 32 lookups with arbitrary s never collide on a bank pair.
+__device__ __forceinline__ void nm_table_replicate(float2* rep, const NmTable* __restrict__ t, int n,
+                                                   int tid, int nthreads)
+{
+    for (int i = tid; i < n * 32; i += nthreads) rep[i] = t->kb[i >> 5];
+}
+
+__device__ __forceinline__ float nm_pwl_eval_rep(const float2* rep, int lane, float x, float inv_h,
+                                                 float off, float nm1, int* idx_out = nullptr)
+{
+    int s = nm_pwl_index(x, inv_h, off, nm1);
+    if (idx_out) *idx_out = s;
+    float2 kb = rep[s * 32 + lane];
+    return __fmaf_rn(kb.x, x, kb.y);
+}
+
+// ---------------------------------------------------------------- dtypes ------
+
+template <typename T> struct NmType;
+template <> struct NmType<float> {
+    static __device__ __forceinline__ float to_f(float v) { return v; }
+    static __device__ __forceinline__ float from_f(float v) { return v; }
+};
+template <> struct NmType<__nv_bfloat16> {
+    static __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+    static __device__ __forceinline__ __nv_bfloat16 from_f(float v) { return __float2bfloat16_rn(v); }
+};
+template <> struct NmType<__half> {
+    static __device__ __forceinline__ float to_f(__half v) { return __half2float(v); }
+    static __device__ __forceinline__ __half from_f(float v) { return __float2half_rn(v); }
+};
+
+__device__ __forceinline__ int8_t nm_quant_i8(float y, float inv_scale)
+{
+    float r = rintf(y * inv_scale);
+    r = fminf(fmaxf(r, -127.0f), 127.0f);
+    return (int8_t)(int)r;
+}
+
+// ---------------------------------------------------------------- PTX ---------
+
+#define NM_WAIT_LIMIT_CYCLES (4000000000LL)  // ~2 s at 2 GHz: every device wait gives up after this
+
+__device__ __forceinline__ uint32_t nm_smem_u32(const void* p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void nm_mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(nm_smem_u32(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void nm_mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(nm_smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void nm_mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(nm_smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ bool nm_mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(nm_smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait on an mbarrier phase.  Gives up when another thread of the CTA has
+// already given up (*abort_flag != 0) or after NM_WAIT_LIMIT_CYCLES; on expiry it
+// records NM_ERR_TIMEOUT in the global status word, raises the CTA's abort flag
+// and returns false.  The caller then skips its remaining work and falls through
+// to the common teardown (no trap, no endless spin).
+__device__ __forceinline__ bool nm_mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                             int* status)
+{
+    if (nm_mbar_try_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    uint32_t spins = 0;
+    while (true) {
+        if (nm_mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > NM_WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, (int)NM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void nm_fence_barrier_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void nm_fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// TMA: 2-D tiled load global -> shared, completion counted on an mbarrier.  c0 is
+// the innermost (contiguous) coordinate and must be a multiple of 16 bytes.
+__device__ __forceinline__ void nm_tma_load_2d(void* smem_dst, const CUtensorMap* tmap, int c0, int c1,
+                                               uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(nm_smem_u32(smem_dst)), "l"(tmap), "r"(nm_smem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void nm_tma_load_3d(void* smem_dst, const CUtensorMap* tmap, int c0, int c1, int c2,
+                                               uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(nm_smem_u32(smem_dst)), "l"(tmap), "r"(nm_smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+__device__ __forceinline__ void nm_prefetch_tmap(const CUtensorMap* tmap)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
+}
+
+// ---- tcgen05 ------------------------------------------------------------------
+
+__device__ __forceinline__ void nm_tmem_alloc(uint32_t* smem_slot, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(nm_smem_u32(smem_slot)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void nm_tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void nm_tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void nm_tc_fence_before()
+{
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void nm_tc_fence_after()
+{
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+// All tcgen05.mma issued so far by this thread arrive (once) on `bar` when done.
+__device__ __forceinline__ void nm_tc_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                     nm_smem_u32(bar))
+                 : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]; kind::f16 covers bf16 and fp16 inputs.
+__device__ __forceinline__ void nm_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void nm_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Shared-memory operand descriptor, 128-byte swizzle, rows of 128 bytes, groups of
+// 8 rows 1024 bytes apart.  Valid for a K-major operand whose K extent per tile is
+// 128 bytes, and for an MN-major operand whose MN extent is 128 bytes (then the
+// 8-row groups run along K).
+__device__ __forceinline__ uint64_t nm_smem_desc_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);       // start address
+    d |= (uint64_t)1 << 16;                             // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                   // stride byte offset: 8 rows * 128 B
+    d |= (uint64_t)1 << 46;                             // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                             // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: D format (1 = f32, 2 = s32), A/B format (f16 kinds:
+// 0 = f16, 1 = bf16; i8 kind: 1 = signed), major-ness (0 = K-major), N>>3, M>>4.
+__host__ __device__ constexpr uint32_t nm_idesc(uint32_t c_fmt, uint32_t ab_fmt, uint32_t a_mn_major,
+                                                uint32_t b_mn_major, uint32_t M, uint32_t N)
+{
+    return (c_fmt << 4) | (ab_fmt << 7) | (ab_fmt << 10) | (a_mn_major << 15) | (b_mn_major << 16) |
+           ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+// 32 lanes x 32 consecutive 32-bit columns of tensor memory into registers: thread
+// l of the warp receives row (lane base + l).
+__device__ __forceinline__ void nm_tmem_ld32(uint32_t taddr, uint32_t* r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void nm_tmem_ld_wait()
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---------------------------------------------------------------- host --------
+
+#define NM_CUDA_TRY(expr)                         \
+    do {                                          \
+        cudaError_t _e = (expr);                  \
+        if (_e != cudaSuccess) return NM_ERR_CUDA; \
+    } while (0)
+
+static inline bool nm_aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
+static inline size_t nm_dtype_size(nm_dtype t)
+{
+    switch (t) {
+    case NM_F32: return 4;
+    case NM_BF16: return 2;
+    case NM_F16: return 2;
+    case NM_I8: return 1;
+    }
+    return 0;
+}
+
+// kernels implemented in the other translation units
+nm_status nm_launch_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int64_t count, nm_dtype dtype,
+                              int32_t* idx_out, cudaStream_t st);
+nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
+                              int64_t rows, int32_t H, float eps, int32_t slot, nm_dtype dtype, cudaStream_t st);
+nm_status nm_launch_quantize(nm_ctx* ctx, const void* x, nm_dtype dtype, int64_t count, float inv_scale,
+                             int8_t* q, cudaStream_t st);
+nm_status nm_launch_linear_simt(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st);
+nm_status nm_launch_linear_tc(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st);
+bool nm_linear_tc_supported(const nm_linear_desc* d);
+nm_status nm_launch_attention_simt(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
+nm_status nm_launch_attention_tc(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
+bool nm_attention_tc_supported(const nm_attn_desc* d);

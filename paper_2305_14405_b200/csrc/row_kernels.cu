@@ -1,0 +1,248 @@
+// HBM-bound kernels of the PWL forward pass: element-wise table evaluation,
+// LayerNorm with PWL rsqrt, and int8 quantisation.  One read and one write per
+// element, 128-bit accesses, no staging through shared memory needed.
+#include "nm_common.cuh"
+
+namespace {
+
+template <typename T, int VEC> struct Pack {
+    T v[VEC];
+};
+
+template <typename T> struct VecOf { static constexpr int N = 16 / sizeof(T); };
+
+template <typename T>
+__device__ __forceinline__ void load16(const T* p, float* f)
+{
+    constexpr int N = VecOf<T>::N;
+    uint4 raw = *reinterpret_cast<const uint4*>(p);
+    const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+    for (int i = 0; i < N; ++i) f[i] = NmType<T>::to_f(e[i]);
+}
+
+template <typename T>
+__device__ __forceinline__ void store16(T* p, const float* f)
+{
+    constexpr int N = VecOf<T>::N;
+    uint4 raw;
+    T* e = reinterpret_cast<T*>(&raw);
+#pragma unroll
+    for (int i = 0; i < N; ++i) e[i] = NmType<T>::from_f(f[i]);
+    *reinterpret_cast<uint4*>(p) = raw;
+}
+
+// ---- y = k[s]*x + b[s] element-wise (Section 3.2: S, then Y = X.K + B) ----------
+template <typename T>
+__global__ void __launch_bounds__(256) pwl_apply_kernel(const NmTable* __restrict__ tab, const T* __restrict__ x,
+                                                        T* __restrict__ y, int64_t count,
+                                                        int32_t* __restrict__ idx_out)
+{
+    extern __shared__ float2 rep[];
+    const int n = tab->n;
+    const float inv_h = tab->inv_h, off = tab->off, nm1 = (float)(n - 1);
+    nm_table_replicate(rep, tab, n, threadIdx.x, blockDim.x);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    constexpr int N = VecOf<T>::N;
+    const int64_t nvec = count / N;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+        float f[N];
+        int s[N];
+        load16<T>(x + v * N, f);
+#pragma unroll
+        for (int i = 0; i < N; ++i) f[i] = nm_pwl_eval_rep(rep, lane, f[i], inv_h, off, nm1, &s[i]);
+        store16<T>(y + v * N, f);
+        if (idx_out) {
+#pragma unroll
+            for (int i = 0; i < N; i += 4)
+                *reinterpret_cast<int4*>(idx_out + v * N + i) = make_int4(s[i], s[i + 1], s[i + 2], s[i + 3]);
+        }
+    }
+    // ragged tail (count not a multiple of the vector width)
+    if (blockIdx.x == 0) {
+        for (int64_t i = nvec * N + threadIdx.x; i < count; i += blockDim.x) {
+            int s;
+            float r = nm_pwl_eval_rep(rep, lane, NmType<T>::to_f(x[i]), inv_h, off, nm1, &s);
+            y[i] = NmType<T>::from_f(r);
+            if (idx_out) idx_out[i] = s;
+        }
+    }
+}
+
+// ---- LayerNorm with PWL rsqrt: one warp per row, the row kept in registers ------
+//   mu = mean(z); v = mean((z-mu)^2); r = PWL_rsqrt(v + eps); y = (z-mu)*r*gamma + beta
+template <typename T, int ITERS>
+__global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restrict__ tab, const T* __restrict__ x,
+                                                        const float* __restrict__ gamma,
+                                                        const float* __restrict__ beta, T* __restrict__ y,
+                                                        int64_t rows, int H, float eps)
+{
+    constexpr int N = VecOf<T>::N;
+    const int lane = threadIdx.x & 31;
+    const int warps_per_block = blockDim.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const T* xr = x + row * H;
+    T* yr = y + row * H;
+    const int nvec = H / N;  // H is a multiple of N
+    float f[ITERS][N];
+    float sum = 0.f;
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        int v = it * 32 + lane;
+        if (v < nvec) {
+            load16<T>(xr + v * N, f[it]);
+#pragma unroll
+            for (int i = 0; i < N; ++i) sum += f[it][i];
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float mu = sum / (float)H;
+    float sq = 0.f;
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        int v = it * 32 + lane;
+        if (v < nvec) {
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+                float dlt = f[it][i] - mu;
+                f[it][i] = dlt;
+                sq = __fmaf_rn(dlt, dlt, sq);
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    const float var = sq / (float)H + eps;
+    const int s = nm_pwl_index(var, tab->inv_h, tab->off, (float)(tab->n - 1));
+    const float2 kb = tab->kb[s];
+    const float r = __fmaf_rn(kb.x, var, kb.y);
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        int v = it * 32 + lane;
+        if (v < nvec) {
+            float g[N], b[N];
+#pragma unroll
+            for (int i = 0; i < N; i += 4) {
+                *reinterpret_cast<float4*>(&g[i]) = __ldg(reinterpret_cast<const float4*>(gamma + v * N + i));
+                *reinterpret_cast<float4*>(&b[i]) = __ldg(reinterpret_cast<const float4*>(beta + v * N + i));
+            }
+#pragma unroll
+            for (int i = 0; i < N; ++i) f[it][i] = __fmaf_rn(f[it][i] * r, g[i], b[i]);
+            store16<T>(yr + v * N, f[it]);
+        }
+    }
+}
+
+// ---- symmetric int8 quantisation with a static scale -----------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) quantize_kernel(const T* __restrict__ x, int64_t count, float inv_scale,
+                                                       int8_t* __restrict__ q)
+{
+    // 16 elements per thread: one or more 16-byte loads, one 16-byte store
+    const int64_t nchunk = count / 16;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    constexpr int N = VecOf<T>::N;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < nchunk; c += stride) {
+        float f[16];
+#pragma unroll
+        for (int i = 0; i < 16; i += N) load16<T>(x + c * 16 + i, f + i);
+        uint4 raw;
+        int8_t* e = reinterpret_cast<int8_t*>(&raw);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) e[i] = nm_quant_i8(f[i], inv_scale);
+        *reinterpret_cast<uint4*>(q + c * 16) = raw;
+    }
+    if (blockIdx.x == 0) {
+        for (int64_t i = nchunk * 16 + threadIdx.x; i < count; i += blockDim.x)
+            q[i] = nm_quant_i8(NmType<T>::to_f(x[i]), inv_scale);
+    }
+}
+
+template <typename T>
+nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const void* x, const float* gamma, const float* beta, void* y,
+                    int64_t rows, int H, float eps, cudaStream_t st)
+{
+    constexpr int N = VecOf<T>::N;
+    const int nvec = H / N;
+    const int iters = (nvec + 31) / 32;
+    const int threads = 256;
+    const int64_t blocks = (rows + 7) / 8;
+    if (blocks > 0x7fffffffLL) return NM_ERR_SHAPE;
+ NmLaunchScope scope(ctx, NM_KERNEL_LAYERNORM, 2.0 * (double)rows * H * sizeof(T), st);
+#define NM_LN_CASE(I)                                                                                      \
+    layernorm_kernel<T, I><<<(unsigned)blocks, threads, 0, st>>>(tab, (const T*)x, gamma, beta, (T*)y, rows, H, eps)
+    if (iters <= 1) NM_LN_CASE(1);
+    else if (iters <= 2) NM_LN_CASE(2);
+    else if (iters <= 3) NM_LN_CASE(3);
+    else if (iters <= 4) NM_LN_CASE(4);
+    else if (iters <= 8) NM_LN_CASE(8);
+    else if (iters <= 16) NM_LN_CASE(16);
+    else return NM_ERR_UNSUPPORTED;
+#undef NM_LN_CASE
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+}  // namespace
+
+nm_status nm_launch_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int64_t count, nm_dtype dtype,
+                              int32_t* idx_out, cudaStream_t st)
+{
+    const NmTable* tab = ctx->d_tables + slot;
+    const int n = ctx->h_tables[slot].n;
+    const size_t smem = (size_t)n * 32 * sizeof(float2);
+    const int threads = 256;
+    int64_t want = (count / 8 + threads - 1) / threads;
+    int blocks = (int)(want < 1 ? 1 : (want > (int64_t)ctx->sm_count * 8 ? (int64_t)ctx->sm_count * 8 : want));
+    NmLaunchScope scope(ctx, NM_KERNEL_PWL_APPLY, 2.0 * (double)count * nm_dtype_size(dtype), st);
+    switch (dtype) {
+    case NM_F32:
+        cudaFuncSetAttribute(pwl_apply_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+        pwl_apply_kernel<float><<<blocks, threads, smem, st>>>(tab, (const float*)x, (float*)y, count, idx_out);
+        break;
+    case NM_BF16:
+        cudaFuncSetAttribute(pwl_apply_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+        pwl_apply_kernel<__nv_bfloat16>
+            <<<blocks, threads, smem, st>>>(tab, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, count, idx_out);
+        break;
+    case NM_F16:
+        cudaFuncSetAttribute(pwl_apply_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+        pwl_apply_kernel<__half><<<blocks, threads, smem, st>>>(tab, (const __half*)x, (__half*)y, count, idx_out);
+        break;
+    default: return NM_ERR_UNSUPPORTED;
+    }
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
+                              int64_t rows, int32_t H, float eps, int32_t slot, nm_dtype dtype, cudaStream_t st)
+{
+    const NmTable* tab = ctx->d_tables + slot;
+    switch (dtype) {
+    case NM_F32: return launch_ln<float>(ctx, tab, x, gamma, beta, y, rows, H, eps, st);
+    case NM_BF16: return launch_ln<__nv_bfloat16>(ctx, tab, x, gamma, beta, y, rows, H, eps, st);
+    case NM_F16: return launch_ln<__half>(ctx, tab, x, gamma, beta, y, rows, H, eps, st);
+    default: return NM_ERR_UNSUPPORTED;
+    }
+}
+
+nm_status nm_launch_quantize(nm_ctx* ctx, const void* x, nm_dtype dtype, int64_t count, float inv_scale,
+                             int8_t* q, cudaStream_t st)
+{
+    const int threads = 256;
+    int64_t want = (count / 16 + threads - 1) / threads;
+    int blocks = (int)(want < 1 ? 1 : (want > (int64_t)ctx->sm_count * 16 ? (int64_t)ctx->sm_count * 16 : want));
+    NmLaunchScope scope(ctx, NM_KERNEL_QUANTIZE, (double)count * (nm_dtype_size(dtype) + 1), st);
+    switch (dtype) {
+    case NM_F32: quantize_kernel<float><<<blocks, threads, 0, st>>>((const float*)x, count, inv_scale, q); break;
+    case NM_BF16:
+        quantize_kernel<__nv_bfloat16><<<blocks, threads, 0, st>>>((const __nv_bfloat16*)x, count, inv_scale, q);
+        break;
+    case NM_F16: quantize_kernel<__half><<<blocks, threads, 0, st>>>((const __half*)x, count, inv_scale, q); break;
+    default: return NM_ERR_UNSUPPORTED;
+    }
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}

@@ -1,0 +1,90 @@
+"""GPU parity, attention with PWL softmax (final row maximum, PWL exp, PWL reciprocal)."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs
+import oracle
+from util import assert_close_bf16, assert_close_f32, load_tables_both, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx(nm):
+    c = nm.Context(0)
+    yield c
+    c.close()
+
+
+def ranges(L):
+    return {"exp": (-8.0, 0.0), "recip": (L / 16.0, float(L))}
+
+
+def run(nm, ctx, dtype, B, L, h, d, algo, seed=0, n=64, qk_scale=1.0):
+    tabs = load_tables_both(ctx, n, ranges(L))
+    H = h * d
+    qkv = nm_inputs.matrix((B * L, 3 * H), seed, dtype, 1.0)
+    qkv[:, :2 * H] *= qk_scale
+    qkv = nm_inputs.round_to(qkv, dtype)
+    td = nm_inputs.torch_dtype(dtype)
+    qd = torch.from_numpy(qkv).cuda().to(td)
+    out = torch.full((B * L, H), float("nan"), dtype=td, device="cuda")
+    ctx.attention_pwl(qd, out, B, L, h, d, algo=algo)
+    ctx.check_device_status()
+    ref = oracle.attention(qkv, B, L, h, d, tabs["exp"], tabs["recip"])
+    return to_np(out), ref
+
+
+@pytest.mark.parametrize("B,L,h,d", [(1, 128, 4, 64), (2, 40, 3, 16), (1, 7, 1, 8)])
+def test_attention_f32_simt(nm, ctx, B, L, h, d):
+    got, ref = run(nm, ctx, "f32", B, L, h, d, nm.ALGO_AUTO)
+    assert_close_f32(got, ref, "attention f32")
+
+
+@pytest.mark.parametrize("algo", ["simt", "tc"])
+@pytest.mark.parametrize("B,L,h,d,qk", [(2, 128, 12, 64, 0.6), (1, 512, 3, 64, 0.6), (3, 128, 2, 64, 1.5), (1, 256, 2, 64, 1.0),
+                                        (1, 384, 1, 64, 0.8)])
+def test_attention_bf16(nm, ctx, algo, B, L, h, d, qk):
+    """Scores of different spread: near-uniform rows (the synthetic BERT workload) and peaked ones
+    that reach the clamped end segments of the exp table."""
+    a = nm.ALGO_SIMT if algo == "simt" else nm.ALGO_TC
+    try:
+        got, ref = run(nm, ctx, "bf16", B, L, h, d, a, seed=L + h, qk_scale=qk)
+    except nm.NmError as e:
+        if algo == "tc" and e.code == 5 and L not in (128, 512):
+            pytest.skip("tensor-core attention kernel takes L in {128, 512} only")
+        raise
+    assert_close_bf16(got, ref, "attention bf16 %s" % algo)
+
+
+@pytest.mark.parametrize("n", [16, 256])
+def test_attention_bf16_segment_counts(nm, ctx, n):
+    got, ref = run(nm, ctx, "bf16", 1, 128, 2, 64, nm.ALGO_AUTO, seed=3, n=n, qk_scale=0.6)
+    assert_close_bf16(got, ref, "attention n=%d" % n)
+
+
+def test_attention_full_size_sampled(nm, ctx):
+    """B=32, L=512, 12 heads of 64: the launch the benchmark times; three sampled batch entries
+    are checked in full against the oracle."""
+    B, L, h, d = 32, 512, 12, 64
+    tabs = load_tables_both(ctx, 64, ranges(L))
+    H = h * d
+    qkv = nm_inputs.matrix((B * L, 3 * H), 77, "bf16", 0.6)
+    qd = torch.from_numpy(qkv).cuda().bfloat16()
+    out = torch.empty((B * L, H), dtype=torch.bfloat16, device="cuda")
+    ctx.attention_pwl(qd, out, B, L, h, d)
+    ctx.check_device_status()
+    for b in (0, 13, 31):
+        ref = oracle.attention(qkv[b * L:(b + 1) * L], 1, L, h, d, tabs["exp"], tabs["recip"])
+        assert_close_bf16(to_np(out[b * L:(b + 1) * L]), ref, "attention full size, batch %d" % b)
+
+
+def test_attention_argument_errors(nm, ctx):
+    load_tables_both(ctx, 64, ranges(128))
+    q = torch.zeros(128, 192, dtype=torch.bfloat16, device="cuda")
+    o = torch.zeros(128, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(nm.NmError) as ei:
+        ctx.attention_pwl(q, o, 1, 128, 1, 64, exp_slot=12)
+    assert ei.value.code == 4
+    ctx.attention_pwl(q, o, 0, 128, 1, 64)     # empty batch: no-op

@@ -1,0 +1,117 @@
+"""GPU parity, whole encoder layers and stacks against the oracle on the seeded workloads."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs
+import oracle
+from util import assert_close_bf16, assert_close_f32, load_tables_both, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx(nm):
+    c = nm.Context(0)
+    yield c
+    c.close()
+
+
+def build(nm, ctx, cfg, layers_np, algo=0):
+    from paper_2305_14405_b200.harness import EncoderModel
+    return EncoderModel(ctx, cfg, layers_np, algo=algo)
+
+
+@pytest.mark.parametrize("random_affine", [False, True])
+def test_c1_tiny_fp32_layer(nm, ctx, random_affine):
+    """Config 1: batch 1, seq 128, hidden 256, 4 heads, FFN 1024, fp32, seed 0, 64-segment tables."""
+    cfg = nm_inputs.C1
+    tabs = load_tables_both(ctx, cfg.segments, cfg.ranges())
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=0, random_affine=random_affine)
+    m = build(nm, ctx, cfg, layers)
+    y = m.forward(torch.from_numpy(x).cuda())
+    ctx.check_device_status()
+    ref = oracle.encoder_layer(x, layers[0], cfg.B, cfg.L, cfg.heads, tabs, cfg.eps)
+    assert_close_f32(to_np(y), ref, "C1 encoder layer")
+
+
+@pytest.mark.parametrize("algo", [0, 1])
+@pytest.mark.parametrize("random_affine", [False, True])
+def test_c2_bert_base_layer_bf16(nm, ctx, algo, random_affine):
+    """Config 2: batch 8, seq 128, hidden 768, 12 heads, FFN 3072, bf16 with fp32 accumulate."""
+    cfg = nm_inputs.C2
+    tabs = load_tables_both(ctx, cfg.segments, cfg.ranges())
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=0, random_affine=random_affine)
+    m = build(nm, ctx, cfg, layers, algo=algo)
+    y = m.forward(torch.from_numpy(x).cuda().bfloat16())
+    ctx.check_device_status()
+    ref = oracle.encoder_layer(x, layers[0], cfg.B, cfg.L, cfg.heads, tabs, cfg.eps)
+    assert_close_bf16(to_np(y), ref, "C2 encoder layer algo %d" % algo)
+
+
+@pytest.mark.parametrize("n", [16, 64, 256])
+def test_c3_stack_sampled_sequences(nm, ctx, n):
+    """Config 3 in the benchmark's launch configuration (12 layers, batch 32, seq 512, bf16).
+    Sequences are independent, so the oracle runs whole sampled sequences: per layer from the
+    GPU's own bf16 layer input, and end to end through all 12 layers."""
+    cfg = nm_inputs.with_(nm_inputs.C3, segments=n)
+    tabs = load_tables_both(ctx, n, cfg.ranges())
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=0)
+    m = build(nm, ctx, cfg, layers)
+    xd = torch.from_numpy(x).cuda().bfloat16()
+    L = cfg.L
+    # per layer: feed each layer the previous GPU output, compare one sequence per layer
+    cur = xd
+    for li in range(cfg.layers):
+        nxt = m.forward_layer(li, cur)
+        if li in (0, 5, 11):
+            b = (7 * li + 3) % cfg.B
+            xin = to_np(cur[b * L:(b + 1) * L])
+            ref = oracle.encoder_layer(xin, layers[li], 1, L, cfg.heads, tabs, cfg.eps)
+            assert_close_bf16(to_np(nxt[b * L:(b + 1) * L]), ref, "C3 layer %d, sequence %d, n=%d" % (li, b, n))
+        cur = nxt
+    ctx.check_device_status()
+    # end to end in one call; must equal the layer-by-layer result bit for bit
+    y = m.forward(xd)
+    ctx.check_device_status()
+    assert torch.equal(y, cur)
+    if n == 64:
+        b = 17
+        ref = oracle.encoder_stack(x[b * L:(b + 1) * L], layers, 1, L, cfg.heads, tabs, cfg.eps)
+        got = to_np(y[b * L:(b + 1) * L])
+        err = np.abs(got - ref)
+        bound = 1e-2 + 1e-2 * np.abs(ref)
+        frac = float((err > bound).mean())
+        # bf16 storage rounding compounds over 12 layers against an fp64 oracle: report, bound loosely
+        print("C3 end-to-end: max err %.4f, fraction outside per-element bound %.5f" % (err.max(), frac))
+        assert frac < 0.02 and err.max() < 0.1
+
+
+def test_encoder_host_entry_point(nm, ctx):
+    cfg = nm_inputs.with_(nm_inputs.C2, B=2)
+    load_tables_both(ctx, cfg.segments, cfg.ranges())
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=1, layers=2)
+    m = build(nm, ctx, cfg, layers)
+    xh = torch.from_numpy(x).bfloat16().pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    xd = torch.empty(xh.shape, dtype=torch.bfloat16, device="cuda")
+    yd = torch.empty_like(xd)
+    ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, xh, yh, xd, yd, m.workspace)
+    y = m.forward(xh.cuda())
+    torch.cuda.synchronize()
+    assert torch.equal(yh, y.cpu())
+
+
+def test_encoder_workspace_errors(nm, ctx):
+    cfg = nm_inputs.with_(nm_inputs.C2, B=1)
+    load_tables_both(ctx, cfg.segments, cfg.ranges())
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=1)
+    m = build(nm, ctx, cfg, layers)
+    xd = torch.from_numpy(x).cuda().bfloat16()
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(nm.NmError) as ei:
+        ctx.encoder_layer(m.structs[0], m.ccfg, xd, torch.empty_like(xd), small)
+    assert ei.value.code == 8
+    with pytest.raises(nm.NmError) as ei:
+        ctx.encoder_layer(m.structs[0], m.ccfg, xd, xd, m.workspace)
+    assert ei.value.code == 1

@@ -1,0 +1,112 @@
+"""GPU parity, HBM-bound row kernels: table evaluation, LayerNorm, int8 quantisation."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs
+import oracle
+from util import FUNCS, assert_close_bf16, assert_close_f32, load_tables_both, to_np
+
+pytestmark = pytest.mark.gpu
+
+RANGES = {"gelu": (-4.0, 4.0), "exp": (-8.0, 0.0), "recip": (8.0, 128.0), "rsqrt": (0.25, 4.0), "relu": (-3.0, 3.0)}
+
+
+@pytest.fixture(scope="module")
+def ctx(nm):
+    c = nm.Context(0)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("name", list(RANGES))
+@pytest.mark.parametrize("n", [2, 16, 64, 256])
+def test_pwl_apply_f32_bit_exact(nm, ctx, name, n):
+    """Segment numbers and fp32 values are bit-exact: both sides take the index with one fp32
+    fused multiply-add and evaluate fma(k, x, b)."""
+    lo, hi = RANGES[name]
+    tabs = load_tables_both(ctx, n, {name: (lo, hi)})
+    x = nm_inputs.pwl_probe_points(lo, hi, n, 100003, seed=n)   # ragged count
+    xd = torch.from_numpy(x).cuda()
+    yd = torch.empty_like(xd)
+    idx = torch.empty(x.size, dtype=torch.int32, device="cuda")
+    from util import SLOTS
+    ctx.pwl_apply(SLOTS[name], xd, yd, idx)
+    ctx.check_device_status()
+    y_ref, idx_ref = oracle.pwl_eval_f32(tabs[name], x)
+    assert np.array_equal(idx.cpu().numpy(), idx_ref)
+    got = yd.cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), y_ref.view(np.uint32))
+
+
+def test_pwl_apply_nan_and_empty(nm, ctx):
+    load_tables_both(ctx, 64, {"gelu": RANGES["gelu"]})
+    x = torch.tensor([float("nan"), 1.0, float("nan"), -2.0, 0.5, 0.25, 8.0, -8.0], device="cuda")
+    y = torch.empty_like(x)
+    idx = torch.empty(8, dtype=torch.int32, device="cuda")
+    ctx.pwl_apply(nm.SLOT_GELU, x, y, idx)
+    assert idx[0].item() == 0 and torch.isnan(y[0]) and idx[2].item() == 0
+    e = torch.empty(0, device="cuda")
+    ctx.pwl_apply(nm.SLOT_GELU, e, e)          # zero elements: a no-op, not an error
+    with pytest.raises(nm.NmError) as ei:
+        ctx.pwl_apply(9, x, y)                 # slot never loaded
+    assert ei.value.code == 4
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+def test_pwl_apply_half_types(nm, ctx, dtype):
+    tabs = load_tables_both(ctx, 64, {"gelu": RANGES["gelu"]})
+    x = nm_inputs.round_to(nm_inputs.matrix((1 << 16) + 24, 3, "f32", 2.0), dtype)
+    td = nm_inputs.torch_dtype(dtype)
+    xd = torch.from_numpy(x).cuda().to(td)
+    yd = torch.empty_like(xd)
+    idx = torch.empty(x.size, dtype=torch.int32, device="cuda")
+    ctx.pwl_apply(nm.SLOT_GELU, xd, yd, idx)
+    y_ref, idx_ref = oracle.pwl_eval_f32(tabs["gelu"], x)
+    assert np.array_equal(idx.cpu().numpy(), idx_ref)
+    want = torch.from_numpy(y_ref).to(td)       # the same fp32 value, rounded to the storage type
+    assert torch.equal(yd.cpu(), want)
+
+
+@pytest.mark.parametrize("dtype,rows,H", [("f32", 128, 256), ("f32", 77, 1000), ("bf16", 1024, 768), ("bf16", 333, 1024),
+                                          ("bf16", 64, 4096), ("f16", 100, 768), ("bf16", 5, 8)])
+def test_layernorm_parity(nm, ctx, dtype, rows, H):
+    tabs = load_tables_both(ctx, 64, {"rsqrt": RANGES["rsqrt"]})
+    rng = np.random.default_rng(rows + H)
+    z = nm_inputs.round_to((rng.standard_normal((rows, H)) * rng.uniform(0.6, 1.8, (rows, 1)) + 0.3).astype(np.float32), dtype)
+    g = (1 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    b = (0.1 * rng.standard_normal(H)).astype(np.float32)
+    td = nm_inputs.torch_dtype(dtype)
+    zd = torch.from_numpy(z).cuda().to(td)
+    yd = torch.empty_like(zd)
+    ctx.layernorm_pwl(zd, torch.from_numpy(g).cuda(), torch.from_numpy(b).cuda(), yd, eps=1e-5)
+    ref = oracle.layernorm(z, g, b, 1e-5, tabs["rsqrt"])
+    if dtype == "f32":
+        assert_close_f32(to_np(yd), ref, "layernorm f32")
+    else:
+        assert_close_bf16(to_np(yd), ref, "layernorm " + dtype)
+
+
+def test_layernorm_rejects_bad_shapes(nm, ctx):
+    load_tables_both(ctx, 64, {"rsqrt": RANGES["rsqrt"]})
+    z = torch.zeros(4, 12, device="cuda")
+    g = torch.ones(12, device="cuda")
+    with pytest.raises(nm.NmError) as ei:
+        ctx.layernorm_pwl(z, g, g, torch.empty_like(z))
+    assert ei.value.code == 2
+    z0 = torch.zeros(0, 16, device="cuda")
+    g16 = torch.ones(16, device="cuda")
+    ctx.layernorm_pwl(z0, g16, g16, torch.empty_like(z0))    # zero rows: no-op
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_quantize_bit_exact(nm, ctx, dtype):
+    x = nm_inputs.round_to(nm_inputs.matrix(70001, 11, "f32", 1.0), dtype)
+    x[:8] = [0.5, 1.5, 2.5, -0.5, -1.5, 1e6, -1e6, 0.0]
+    x = nm_inputs.round_to(x, dtype)
+    scale = np.float32(0.03)
+    inv = float(np.float32(1.0) / scale)
+    xd = torch.from_numpy(x).cuda().to(nm_inputs.torch_dtype(dtype))
+    q = torch.empty(x.size, dtype=torch.int8, device="cuda")
+    ctx.quantize_i8(xd, inv, q)
+    assert np.array_equal(q.cpu().numpy(), oracle.quantize_i8(x, scale))

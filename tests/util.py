@@ -1,0 +1,56 @@
+"""Shared checks for the GPU parity tests."""
+import numpy as np
+import torch
+
+# bf16 / fp16 paths: |gpu - oracle| <= 1e-2 + 1e-2*|oracle| per element
+BF16_ATOL, BF16_RTOL = 1e-2, 1e-2
+# fp32 path: |gpu - oracle| <= 1e-4 * max(|oracle|, rms(oracle))
+F32_RTOL = 1e-4
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu").to(torch.float64).numpy() if t.dtype != torch.int8 and t.dtype != torch.int32 \
+        else t.detach().to("cpu").numpy()
+
+
+def assert_close_bf16(gpu, ref, what=""):
+    gpu = np.asarray(gpu, np.float64)
+    ref = np.asarray(ref, np.float64)
+    assert gpu.shape == ref.shape, (gpu.shape, ref.shape)
+    assert np.all(np.isfinite(gpu)), what + ": non-finite GPU output"
+    err = np.abs(gpu - ref)
+    bound = BF16_ATOL + BF16_RTOL * np.abs(ref)
+    bad = err > bound
+    assert not bad.any(), "%s: %d / %d elements outside 1e-2 + 1e-2*|ref| (max err %.3e at ref %.3e)" % (
+        what, bad.sum(), bad.size, err.max(), ref.ravel()[err.argmax()])
+
+
+def assert_close_f32(gpu, ref, what="", rtol=F32_RTOL):
+    gpu = np.asarray(gpu, np.float64)
+    ref = np.asarray(ref, np.float64)
+    assert gpu.shape == ref.shape
+    assert np.all(np.isfinite(gpu)), what + ": non-finite GPU output"
+    rms = np.sqrt(np.mean(ref * ref))
+    bound = rtol * np.maximum(np.abs(ref), rms)
+    err = np.abs(gpu - ref)
+    bad = err > bound
+    assert not bad.any(), "%s: %d / %d elements outside %.0e*max(|ref|, rms) (max err %.3e, rms %.3e)" % (
+        what, bad.sum(), bad.size, rtol, err.max(), rms)
+
+
+FUNCS = {"gelu": 0, "exp": 1, "recip": 2, "rsqrt": 3, "relu": 4, "sqrt": 5, "identity": 6}
+SLOTS = {"gelu": 0, "exp": 1, "recip": 2, "rsqrt": 3, "relu": 4}
+
+
+def load_tables_both(ctx, n, ranges):
+    """Builds each table twice -- by the library's builder and by the oracle's -- checks they
+    agree bit for bit, loads the library's into the context and returns the oracle's."""
+    import oracle
+    out = {}
+    for name, (lo, hi) in ranges.items():
+        k, b = ctx.load_function_table(SLOTS[name], FUNCS[name], n, lo, hi)
+        t = oracle.Table.secant(FUNCS[name], n, lo, hi)
+        assert np.array_equal(np.asarray(k, np.float32), t.k), name
+        assert np.array_equal(np.asarray(b, np.float32), t.b), name
+        out[name] = t
+    return out
