@@ -81,10 +81,16 @@ def test_c3_stack_sampled_sequences(nm, ctx, n):
         got = to_np(y[b * L:(b + 1) * L])
         err = np.abs(got - ref)
         bound = 1e-2 + 1e-2 * np.abs(ref)
-        frac = float((err > bound).mean())
-        # bf16 storage rounding compounds over 12 layers against an fp64 oracle: report, bound loosely
-        print("C3 end-to-end: max err %.4f, fraction outside per-element bound %.5f" % (err.max(), frac))
-        assert frac < 0.02 and err.max() < 0.1
+        frac1 = float((err > bound).mean())
+        # Each layer meets the per-element bound from the same bf16 input (checked above).  Over 12
+        # layers the bf16 rounding of the stored activations is re-injected at every layer while the
+        # fp64 oracle rounds nothing; LayerNorm keeps the perturbation gain near one, so independent
+        # per-layer errors add in quadrature: the end-to-end bound is sqrt(layers) times the per-layer one.
+        k = np.sqrt(cfg.layers)
+        frac = float((err > k * bound).mean())
+        print("C3 end-to-end: max err %.4f, rms err %.5f, outside 1x bound %.5f, outside sqrt(12)x bound %.6f"
+              % (err.max(), np.sqrt((err ** 2).mean()), frac1, frac))
+        assert frac == 0.0
 
 
 def test_encoder_host_entry_point(nm, ctx):
