@@ -12,8 +12,9 @@
 //   warp 0      one lane: TMA loads of Q, K, V (128-byte swizzle), tcgen05.mma for
 //               S = Q K^T (K-major operands) and O += P V (V as an MN-major operand,
 //               straight from its [keys, d] layout), commits on mbarriers
-//   warps 1-4   one thread per query row: tcgen05.ld of S, row maximum and row sum with
-//               no shuffles at all, PWL exp from a per-lane replicated table, P written
+//   warps 1-8   two threads per query row (each owns every other 64-key chunk): tcgen05.ld
+//               of S, row maximum and row sum without shuffles (one exchange through shared
+//               memory), PWL exp from a per-lane replicated table, P written
 //               to shared memory as bf16 in the swizzled K-major layout the MMA reads,
 //               PWL reciprocal, final scaling and store.
 // For L = 512 the S block fills all 512 tensor-memory columns; O then reuses columns
@@ -25,7 +26,7 @@ namespace {
 constexpr int BQ = 128;          // query rows per CTA
 constexpr int HD = 64;           // head dimension
 constexpr int ROWB = 128;        // bytes per tile row (64 x 16-bit)
-constexpr int NTHREADS = 160;
+constexpr int NTHREADS = 288;   // warp 0: TMA + MMA; warps 1-8: softmax
 constexpr int MAX_PBUF = 4;
 
 struct AttnArgs {
@@ -73,6 +74,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __shared__ uint64_t bar_p_full[MAX_PBUF], bar_p_empty[MAX_PBUF];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float s_red[2][BQ];   // row maximum / row sum exchange between the two halves
 
     const int L = a.L;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -169,7 +171,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
         }
     } else {
+        // ---- softmax warps: two per tensor-memory lane quarter.  Half h of a quarter owns the
+        // 64-key chunks c with (c & 1) == h in both passes; row maximum and row sum are
+        // combined across the two halves through shared memory.
         const int q = warp & 3;
+        const int h = (warp - 1) >> 2;
         const int row = q * 32 + lane;
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
         const float inv_h = a.t_exp->inv_h, off = a.t_exp->off, nm1 = (float)(a.n_exp - 1);
@@ -178,23 +184,36 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         int ok = 1;
         if (lane == 0) ok = nm_mbar_wait(&bar_s, 0, abortp, a.status) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
+        float m = -INFINITY;
         if (ok) {
             nm_tc_fence_after();
-            // ---- pass 1: final row maximum (thread-local: one thread owns the row)
-            float m = -INFINITY;
+            // ---- pass 1: maximum over this warp's chunks (thread-local: one thread, one row)
 #pragma unroll 1
-            for (int c = 0; c < L / 32; ++c) {
-                uint32_t r[32];
-                nm_tmem_ld32(t_row + (uint32_t)(c * 32), r);
-                nm_tmem_ld_wait();
+            for (int c = h; c < n_pchunks; c += 2) {
+                uint32_t r[64];
+                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64), r);
+                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64 + 32), r + 32);
+                nm_tmem_ld_wait32(r);
+                nm_tmem_ld_wait32(r + 32);
+                float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) m = fmaxf(m, __uint_as_float(r[i]));
+                for (int i = 0; i < 64; i += 2) {
+                    m0 = fmaxf(m0, __uint_as_float(r[i]));
+                    m1 = fmaxf(m1, __uint_as_float(r[i + 1]));
+                }
+                m = fmaxf(m, fmaxf(m0, m1));
             }
-            const float neg_ms = -(m * a.scale);
-            float sum = 0.f;
+        }
+        s_red[h][row] = m;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        m = fmaxf(s_red[0][row], s_red[1][row]);   // the FINAL row maximum
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        const float neg_ms = -(m * a.scale);
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        if (ok) {
             // ---- pass 2: e = PWL_exp(s - m), row sum, P tiles for the second MMA
 #pragma unroll 1
-            for (int c = 0; c < n_pchunks; ++c) {
+            for (int c = h; c < n_pchunks; c += 2) {
                 const int buf = c % a.nbuf;
                 if (c >= a.nbuf) {
                     if (lane == 0) ok = nm_mbar_wait(&bar_p_empty[buf], (uint32_t)(((c / a.nbuf) - 1) & 1), abortp, a.status) ? 1 : 0;
@@ -202,32 +221,29 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (!ok) break;
                 }
                 uint8_t* prow = p_s + (size_t)buf * BQ * ROWB + (size_t)row * ROWB;
+                uint32_t r[64];
+                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64), r);
+                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64 + 32), r + 32);
+                nm_tmem_ld_wait32(r);
+                nm_tmem_ld_wait32(r + 32);
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t r[32];
-                    nm_tmem_ld32(t_row + (uint32_t)(c * 64 + half * 32), r);
-                    nm_tmem_ld_wait();
-                    uint32_t pk[16];
+                for (int j = 0; j < 8; ++j) {   // 8 keys = one 16-byte chunk of the P row
+                    uint32_t pk[4];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float x0 = __fmaf_rn(__uint_as_float(r[i]), a.scale, neg_ms);
-                        const float x1 = __fmaf_rn(__uint_as_float(r[i + 1]), a.scale, neg_ms);
+                    for (int i = 0; i < 4; ++i) {
+                        const float x0 = __fmaf_rn(__uint_as_float(r[j * 8 + 2 * i]), a.scale, neg_ms);
+                        const float x1 = __fmaf_rn(__uint_as_float(r[j * 8 + 2 * i + 1]), a.scale, neg_ms);
                         const int s0 = nm_pwl_index(x0, inv_h, off, nm1);
                         const int s1 = nm_pwl_index(x1, inv_h, off, nm1);
                         const float2 kb0 = rep[(s0 << shift) + copy];
                         const float2 kb1 = rep[(s1 << shift) + copy];
                         const float e0 = __fmaf_rn(kb0.x, x0, kb0.y);
                         const float e1 = __fmaf_rn(kb1.x, x1, kb1.y);
-                        sum += e0;
-                        sum += e1;
-                        pk[i >> 1] = AttnT<T>::pack(e0, e1);
+                        if (i & 1) { sum2 += e0; sum3 += e1; } else { sum0 += e0; sum1 += e1; }
+                        pk[i] = AttnT<T>::pack(e0, e1);
                     }
-                    // 32 keys = 4 chunks of 16 bytes; chunk index is XORed with the row (128-byte swizzle)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int chunk = (half * 4 + j) ^ (row & 7);
-                        *reinterpret_cast<uint4*>(prow + chunk * 16) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                    }
+                    // chunk index is XORed with the row (128-byte swizzle of the K-major P tile)
+                    *reinterpret_cast<uint4*>(prow + ((j ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
                 nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
                 nm_tc_fence_before();
@@ -235,30 +251,30 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (lane == 0) nm_mbar_arrive(&bar_p_full[buf]);
                 __syncwarp();
             }
+        }
+        s_red[h][row] = (sum0 + sum1) + (sum2 + sum3);
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        const float sum = s_red[0][row] + s_red[1][row];
+        if (ok) {
+            // ---- r = PWL_recip(sigma), then O * r; each half stores 32 of the 64 channels
+            const int sr = nm_pwl_index(sum, a.t_rcp->inv_h, a.t_rcp->off, (float)(a.t_rcp->n - 1));
+            const float2 kbr = a.t_rcp->kb[sr];
+            const float rinv = __fmaf_rn(kbr.x, sum, kbr.y);
+            if (lane == 0) ok = nm_mbar_wait(&bar_o, 0, abortp, a.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
             if (ok) {
-                // ---- r = PWL_recip(sigma), then O * r
-                const int sr = nm_pwl_index(sum, a.t_rcp->inv_h, a.t_rcp->off, (float)(a.t_rcp->n - 1));
-                const float2 kbr = a.t_rcp->kb[sr];
-                const float rinv = __fmaf_rn(kbr.x, sum, kbr.y);
-                if (lane == 0) ok = nm_mbar_wait(&bar_o, 0, abortp, a.status) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (ok) {
-                    nm_tc_fence_after();
-                    T* orow = reinterpret_cast<T*>(a.out) + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) + (size_t)g * HD;
+                nm_tc_fence_after();
+                T* orow = reinterpret_cast<T*>(a.out) + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) + (size_t)g * HD + h * 32;
+                uint32_t r[32];
+                nm_tmem_ld32_async(t_row + a.o_col + (uint32_t)(h * 32), r);
+                nm_tmem_ld_wait32(r);
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t r[32];
-                        nm_tmem_ld32(t_row + a.o_col + (uint32_t)(half * 32), r);
-                        nm_tmem_ld_wait();
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t w[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                w[i] = AttnT<T>::pack(__uint_as_float(r[j * 8 + 2 * i]) * rinv, __uint_as_float(r[j * 8 + 2 * i + 1]) * rinv);
-                            reinterpret_cast<uint4*>(orow + half * 32)[j] = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    }
+                    for (int i = 0; i < 4; ++i)
+                        w[i] = AttnT<T>::pack(__uint_as_float(r[j * 8 + 2 * i]) * rinv, __uint_as_float(r[j * 8 + 2 * i + 1]) * rinv);
+                    reinterpret_cast<uint4*>(orow)[j] = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
         }

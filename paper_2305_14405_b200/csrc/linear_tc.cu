@@ -10,8 +10,10 @@
 //   warp 1     tcgen05.mma issuer (one lane); accumulators live in tensor memory,
 //              two buffers of BN columns so the epilogue of tile i overlaps the
 //              main loop of tile i+1
-//   warps 2-5  epilogue: tcgen05.ld -> bias/scale -> segment index -> k*x+b from a
-//              per-lane replicated table in shared memory -> residual -> store.
+//   warps 2-9  epilogue, two warps per tensor-memory lane quarter: tcgen05.ld -> bias/scale ->
+//              segment index -> k*x+b from a per-lane replicated table in shared memory ->
+//              residual -> store; the loads of the next 32-column chunk are in flight
+//              while the current one is computed.
 // The nonlinearity therefore costs no pass over HBM.
 #include "nm_common.cuh"
 
@@ -21,7 +23,7 @@ constexpr int BM = 128;
 constexpr int ROW_BYTES = 128;  // bytes of K per tile row = one swizzle span
 constexpr int A_BYTES = BM * ROW_BYTES;
 constexpr int MAX_STAGES = 8;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, 8 epilogue warps
 
 struct TcArgs {
     int64_t M, N, K;
@@ -97,18 +99,18 @@ template <> __device__ __forceinline__ void store32<int8_t>(int8_t* p, const flo
 template <typename OutT> __device__ __forceinline__ void store1(OutT* p, float v, float) { *p = NmType<OutT>::from_f(v); }
 template <> __device__ __forceinline__ void store1<int8_t>(int8_t* p, float v, float inv) { *p = nm_quant_i8(v, inv); }
 
-template <typename OutT> __device__ __forceinline__ void add_res32(const OutT* p, float* v)
+template <typename OutT> __device__ __forceinline__ void add_res32(const uint4* p, float* v)
 {
     constexpr int PER = 16 / sizeof(OutT);
 #pragma unroll
     for (int q = 0; q < 32 / PER; ++q) {
-        uint4 raw = __ldg(reinterpret_cast<const uint4*>(p) + q);
+        uint4 raw = p[q];
         const OutT* e = reinterpret_cast<const OutT*>(&raw);
 #pragma unroll
         for (int i = 0; i < PER; ++i) v[q * PER + i] += NmType<OutT>::to_f(e[i]);
     }
 }
-template <> __device__ __forceinline__ void add_res32<int8_t>(const int8_t*, float*) {}
+template <> __device__ __forceinline__ void add_res32<int8_t>(const uint4*, float*) {}
 template <typename OutT> __device__ __forceinline__ float res1(const OutT* p) { return NmType<OutT>::to_f(*p); }
 template <> __device__ __forceinline__ float res1<int8_t>(const int8_t*) { return 0.f; }
 
@@ -147,7 +149,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             nm_mbar_init(&bar_acc_full[b], 1);
-            nm_mbar_init(&bar_acc_empty[b], 4);
+            nm_mbar_init(&bar_acc_empty[b], 8);
         }
         nm_mbar_init(&bar_drain, 1);
         nm_fence_barrier_init();
@@ -234,8 +236,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
         }
     } else {
-        // ------------------------------------------------ epilogue (warps 2..5)
-        const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+        // ------------------------------------------------ epilogue (warps 2..9)
+        // Two warps per tensor-memory lane quarter; each takes half of the tile's columns in
+        // 32-column chunks.  The tensor-memory load and the residual load of chunk i+1 are in
+        // flight while chunk i is computed and stored.
+        const int q = warp & 3;              // lane quarter this warp may read
+        const int half = (warp - 2) >> 2;    // which half of the columns
+        constexpr int NCH = BN / 64;         // chunks per warp per tile
+        constexpr int RV = 2 * (int)sizeof(OutT);  // 16-byte vectors of residual per 32 columns
         int buf = 0;
         uint32_t acc_phase = 0;
         const bool has_tab = a.tab != nullptr;
@@ -246,7 +254,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const OutT* res = reinterpret_cast<const OutT*>(a.residual);
         for (int tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x) {
             const int m0 = (tile / a.num_n_tiles) * BM;
-            const int n0 = (tile % a.num_n_tiles) * BN;
+            const int n0 = (tile % a.num_n_tiles) * BN + half * (BN / 2);
             int ok = 1;
             if (lane == 0) ok = nm_mbar_wait(&bar_acc_full[buf], acc_phase, abortp, a.status) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -254,90 +262,104 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             nm_tc_fence_after();
             const int64_t row = (int64_t)m0 + q * 32 + lane;
             const bool row_ok = row < a.M;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                nm_tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
-                nm_tmem_ld_wait();
-                if (c == BN / 32 - 1) {
-                    // accumulator fully read: hand the buffer back to the MMA warp
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2));
+            uint32_t r[2][32];
+            uint4 rs[2][RV];
+            nm_tmem_ld32_async(t_addr, r[0]);
+            if (res && row_ok && n0 + 32 <= a.N) {
+#pragma unroll
+                for (int v = 0; v < RV; ++v) rs[0][v] = __ldg(reinterpret_cast<const uint4*>(res + row * a.ldr + n0) + v);
+            }
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                const int cur = c & 1;
+                nm_tmem_ld_wait32(r[cur]);
+                const int64_t col0 = (int64_t)n0 + c * 32;
+                if (c + 1 < NCH) {
+                    nm_tmem_ld32_async(t_addr + (uint32_t)((c + 1) * 32), r[cur ^ 1]);
+                    if (res && row_ok && col0 + 64 <= a.N) {
+#pragma unroll
+                        for (int v = 0; v < RV; ++v)
+                            rs[cur ^ 1][v] = __ldg(reinterpret_cast<const uint4*>(res + row * a.ldr + col0 + 32) + v);
+                    }
+                } else {
+                    // this warp's share of the accumulator is in registers: hand the buffer back
                     nm_tc_fence_before();
                     __syncwarp();
                     if (lane == 0) nm_mbar_arrive(&bar_acc_empty[buf]);
                     __syncwarp();
                 }
-                const int64_t col0 = (int64_t)n0 + c * 32;
                 // lanes beyond the last row / column skip the arithmetic but stay in the loop:
-                // the tensor-memory loads above need the whole warp
+                // the tensor-memory loads need the whole warp
                 if (row_ok && col0 < a.N) {
-                float v[32];
-                if (col0 + 32 <= a.N) {
-                    if constexpr (TcIn<InT>::is_int) {
-                        if (a.acc_dump) {
+                    float v[32];
+                    if (col0 + 32 <= a.N) {
+                        if constexpr (TcIn<InT>::is_int) {
+                            if (a.acc_dump) {
 #pragma unroll
-                            for (int i = 0; i < 32; i += 4)
-                                *reinterpret_cast<int4*>(a.acc_dump + row * a.N + col0 + i) =
-                                    make_int4((int)r[i], (int)r[i + 1], (int)r[i + 2], (int)r[i + 3]);
-                        }
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4) {
-                            const float4 ws = __ldg(reinterpret_cast<const float4*>(a.w_scale + col0 + i));
-                            float4 bs = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (a.bias) bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
-                            v[i] = __fmaf_rn((float)(int)r[i], a.a_scale * ws.x, bs.x);
-                            v[i + 1] = __fmaf_rn((float)(int)r[i + 1], a.a_scale * ws.y, bs.y);
-                            v[i + 2] = __fmaf_rn((float)(int)r[i + 2], a.a_scale * ws.z, bs.z);
-                            v[i + 3] = __fmaf_rn((float)(int)r[i + 3], a.a_scale * ws.w, bs.w);
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                        if (a.bias) {
+                                for (int i = 0; i < 32; i += 4)
+                                    *reinterpret_cast<int4*>(a.acc_dump + row * a.N + col0 + i) =
+                                        make_int4((int)r[cur][i], (int)r[cur][i + 1], (int)r[cur][i + 2], (int)r[cur][i + 3]);
+                            }
 #pragma unroll
                             for (int i = 0; i < 32; i += 4) {
-                                const float4 bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
-                                v[i] += bs.x; v[i + 1] += bs.y; v[i + 2] += bs.z; v[i + 3] += bs.w;
-                            }
-                        }
-                    }
-                    if (has_tab) {
-                        if (a.idx_dump) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                int s;
-                                v[i] = nm_pwl_eval_rep(rep, lane, v[i], inv_h, off, nm1, &s);
-                                a.idx_dump[row * a.N + col0 + i] = s;
+                                const float4 ws = __ldg(reinterpret_cast<const float4*>(a.w_scale + col0 + i));
+                                float4 bs = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (a.bias) bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
+                                v[i] = __fmaf_rn((float)(int)r[cur][i], a.a_scale * ws.x, bs.x);
+                                v[i + 1] = __fmaf_rn((float)(int)r[cur][i + 1], a.a_scale * ws.y, bs.y);
+                                v[i + 2] = __fmaf_rn((float)(int)r[cur][i + 2], a.a_scale * ws.z, bs.z);
+                                v[i + 3] = __fmaf_rn((float)(int)r[cur][i + 3], a.a_scale * ws.w, bs.w);
                             }
                         } else {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = nm_pwl_eval_rep(rep, lane, v[i], inv_h, off, nm1);
-                        }
-                    }
-                    if (res) add_res32<OutT>(res + row * a.ldr + col0, v);
-                    store32<OutT>(out + row * a.ldo + col0, v, a.inv_out_scale);
-                } else {
-                    // ragged right edge: element by element
+                            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[cur][i]);
+                            if (a.bias) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int64_t col = col0 + i;
-                        if (col >= a.N) continue;
-                        float x;
-                        const float bj = a.bias ? a.bias[col] : 0.f;
-                        if constexpr (TcIn<InT>::is_int) {
-                            if (a.acc_dump) a.acc_dump[row * a.N + col] = (int)r[i];
-                            x = __fmaf_rn((float)(int)r[i], a.a_scale * a.w_scale[col], bj);
-                        } else {
-                            x = __uint_as_float(r[i]) + bj;
+                                for (int i = 0; i < 32; i += 4) {
+                                    const float4 bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
+                                    v[i] += bs.x; v[i + 1] += bs.y; v[i + 2] += bs.z; v[i + 3] += bs.w;
+                                }
+                            }
                         }
                         if (has_tab) {
-                            int s;
-                            x = nm_pwl_eval_rep(rep, lane, x, inv_h, off, nm1, &s);
-                            if (a.idx_dump) a.idx_dump[row * a.N + col] = s;
+                            if (a.idx_dump) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) {
+                                    int s;
+                                    v[i] = nm_pwl_eval_rep(rep, lane, v[i], inv_h, off, nm1, &s);
+                                    a.idx_dump[row * a.N + col0 + i] = s;
+                                }
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) v[i] = nm_pwl_eval_rep(rep, lane, v[i], inv_h, off, nm1);
+                            }
                         }
-                        if (res) x += res1<OutT>(res + row * a.ldr + col);
-                        store1<OutT>(out + row * a.ldo + col, x, a.inv_out_scale);
+                        if (res) add_res32<OutT>(rs[cur], v);
+                        store32<OutT>(out + row * a.ldo + col0, v, a.inv_out_scale);
+                    } else {
+                        // ragged right edge: element by element
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int64_t col = col0 + i;
+                            if (col >= a.N) continue;
+                            float x;
+                            const float bj = a.bias ? a.bias[col] : 0.f;
+                            if constexpr (TcIn<InT>::is_int) {
+                                if (a.acc_dump) a.acc_dump[row * a.N + col] = (int)r[cur][i];
+                                x = __fmaf_rn((float)(int)r[cur][i], a.a_scale * a.w_scale[col], bj);
+                            } else {
+                                x = __uint_as_float(r[cur][i]) + bj;
+                            }
+                            if (has_tab) {
+                                int s;
+                                x = nm_pwl_eval_rep(rep, lane, x, inv_h, off, nm1, &s);
+                                if (a.idx_dump) a.idx_dump[row * a.N + col] = s;
+                            }
+                            if (res) x += res1<OutT>(res + row * a.ldr + col);
+                            store1<OutT>(out + row * a.ldo + col, x, a.inv_out_scale);
+                        }
                     }
-                }
                 }
                 __syncwarp();
             }
@@ -345,6 +367,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (buf == 0) acc_phase ^= 1u;
         }
     }
+
 
     // ---------------------------------------------------- teardown (all paths)
     nm_tc_fence_before();
