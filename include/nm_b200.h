@@ -118,7 +118,8 @@ nm_status nm_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int64_t co
  *   accumulators and the segment numbers, for bit-exact checks.
  * All pointers 16-byte aligned, lda/ldw/ldo/ldr multiples of 16 bytes.
  * algo: 0 = pick; 1 = force the plain SIMT kernel; 2 = force the tcgen05 kernel
- * (NM_ERR_UNSUPPORTED if the shape or dtype has none). */
+ * (NM_ERR_UNSUPPORTED if the shape or dtype has none); 3 = tcgen05 with one CTA per
+ * tile even where the two-CTA (cta_group::2) tile would be chosen. */
 typedef struct {
     int64_t M, N, K;
     nm_dtype in_dtype;

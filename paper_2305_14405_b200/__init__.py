@@ -19,7 +19,7 @@ NM_OK = 0
 F32, BF16, F16, I8 = 0, 1, 2, 3
 SLOT_NONE, SLOT_GELU, SLOT_EXP, SLOT_RECIP, SLOT_RSQRT, SLOT_RELU, SLOT_USER0 = -1, 0, 1, 2, 3, 4, 5
 FUNC_GELU, FUNC_EXP, FUNC_RECIP, FUNC_RSQRT, FUNC_RELU, FUNC_SQRT, FUNC_IDENTITY = range(7)
-ALGO_AUTO, ALGO_SIMT, ALGO_TC = 0, 1, 2
+ALGO_AUTO, ALGO_SIMT, ALGO_TC, ALGO_TC_1CTA = 0, 1, 2, 3
 
 EXPORTS = [
     "nm_status_string", "nm_ctx_create", "nm_ctx_destroy", "nm_ctx_poll_status", "nm_ctx_launch_count",

@@ -13,7 +13,7 @@ OBJ = os.path.join(HERE, "build")
 SO = os.path.join(HERE, "libnm_b200.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-         "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
+         "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"] + os.environ.get("NM_NVCC_EXTRA", "").split()
 
 
 def _sources():

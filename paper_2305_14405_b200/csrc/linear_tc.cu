@@ -5,32 +5,43 @@
 //   out[m][j] = PWL( sum_c A[m][c]*W[j][c] * scale_j + bias[j] ) + residual[m][j]
 //
 // Persistent, warp-specialised kernel, one CTA per SM:
-//   warp 0     TMA producer: 128 x 128-byte A tile and BN x 128-byte W tile per stage,
-//              128-byte swizzle, multi-stage mbarrier ring
-//   warp 1     tcgen05.mma issuer (one lane); accumulators live in tensor memory,
-//              two buffers of BN columns so the epilogue of tile i overlaps the
-//              main loop of tile i+1
-//   warps 2-9  epilogue, two warps per tensor-memory lane quarter: tcgen05.ld -> bias/scale ->
-//              segment index -> k*x+b from a per-lane replicated table in shared memory ->
-//              residual -> store; the loads of the next 32-column chunk are in flight
-//              while the current one is computed.
+//   warp 0     TMA producer: 128 x 128-byte A tile and W tile per stage, 128-byte swizzle,
+//              multi-stage mbarrier ring
+//   warp 1     tcgen05.mma issuer (one lane); accumulators live in tensor memory, two
+//              buffers of 256 columns so the epilogue of tile i overlaps the main loop
+//              of tile i+1
+//   warps 2-9  epilogue, two warps per tensor-memory lane quarter.  Per 32-column chunk:
+//              tcgen05.ld (the next chunk's load in flight) -> bias/scale -> segment index
+//              -> k*x+b from a per-lane replicated table in shared memory -> residual.
+//              Results are staged in shared memory (32 rows x 128 bytes per warp, 128-byte
+//              swizzle) and leave with one TMA store per group, so global writes are whole
+//              lines; the residual arrives the same way through a TMA load that is issued
+//              one group ahead.
 // The nonlinearity therefore costs no pass over HBM.
+//
+// TWO = false: one CTA per 128 x 256 tile (tcgen05 cta_group::1).
+// TWO = true:  a cluster of two CTAs per 256 x 256 tile (cta_group::2): each CTA loads its
+//   own 128 rows of A and its own 128 rows of W, the leader CTA issues one MMA over both,
+//   and each CTA's tensor memory receives its 128 x 256 half of the accumulator.
+#include <string.h>
+
 #include "nm_common.cuh"
 
 namespace {
 
 constexpr int BM = 128;
+constexpr int BN = 256;
 constexpr int ROW_BYTES = 128;  // bytes of K per tile row = one swizzle span
 constexpr int A_BYTES = BM * ROW_BYTES;
 constexpr int MAX_STAGES = 8;
 constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, 8 epilogue warps
+constexpr int NUM_EPI_WARPS = 8;
+constexpr int STAGE_BUF = 32 * 128;  // one staging buffer: 32 rows x 128 bytes
 
 struct TcArgs {
     int64_t M, N, K;
-    int64_t ldr, ldo;
     const float* bias;
-    const void* residual;
-    void* out;
+    int has_res;
     const NmTable* tab;
     float a_scale;
     const float* w_scale;
@@ -39,7 +50,22 @@ struct TcArgs {
     int32_t* idx_dump;
     int* status;
     int num_n_tiles, num_tiles, num_k_blocks, stages, n_seg;
+#ifdef NM_EXP_TIMELINE
+    long long* dbg;  // development only: per-CTA timestamps
+#endif
 };
+#ifdef NM_EXP_TIMELINE
+#include <stdlib.h>
+__device__ __forceinline__ long long nm_gtime()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define NM_TL(slot) do { if (a.dbg && blockIdx.x < 8) a.dbg[blockIdx.x * 64 + (slot)] = nm_gtime(); } while (0)
+#else
+#define NM_TL(slot) do {} while (0)
+#endif
 
 template <typename InT> struct TcIn;
 template <> struct TcIn<__nv_bfloat16> {
@@ -55,162 +81,194 @@ template <> struct TcIn<int8_t> {
     static constexpr bool is_int = true;
 };
 
-template <typename OutT> __device__ __forceinline__ void store32(OutT* p, const float* v, float inv);
-template <> __device__ __forceinline__ void store32<__nv_bfloat16>(__nv_bfloat16* p, const float* v, float)
+// 32 fp32 values -> 32*sizeof(OutT)/4 packed words
+template <typename OutT> __device__ __forceinline__ void pack32(const float* v, uint32_t* w, float inv);
+template <> __device__ __forceinline__ void pack32<__nv_bfloat16>(const float* v, uint32_t* w, float)
 {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint4 raw;
-        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
-        reinterpret_cast<uint4*>(p)[q] = raw;
+    for (int i = 0; i < 16; ++i) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t*>(&h);
     }
 }
-template <> __device__ __forceinline__ void store32<__half>(__half* p, const float* v, float)
+template <> __device__ __forceinline__ void pack32<__half>(const float* v, uint32_t* w, float)
 {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint4 raw;
-        __half2* h = reinterpret_cast<__half2*>(&raw);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
-        reinterpret_cast<uint4*>(p)[q] = raw;
+    for (int i = 0; i < 16; ++i) {
+        __half2 h = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t*>(&h);
     }
 }
-template <> __device__ __forceinline__ void store32<float>(float* p, const float* v, float)
+template <> __device__ __forceinline__ void pack32<float>(const float* v, uint32_t* w, float)
 {
 #pragma unroll
-    for (int q = 0; q < 8; ++q)
-        reinterpret_cast<float4*>(p)[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i]);
 }
-template <> __device__ __forceinline__ void store32<int8_t>(int8_t* p, const float* v, float inv)
+template <> __device__ __forceinline__ void pack32<int8_t>(const float* v, uint32_t* w, float inv)
 {
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
-        uint4 raw;
-        int8_t* e = reinterpret_cast<int8_t*>(&raw);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) e[i] = nm_quant_i8(v[q * 16 + i], inv);
-        reinterpret_cast<uint4*>(p)[q] = raw;
+    for (int i = 0; i < 8; ++i) {
+        uint32_t b0 = (uint8_t)nm_quant_i8(v[4 * i], inv), b1 = (uint8_t)nm_quant_i8(v[4 * i + 1], inv);
+        uint32_t b2 = (uint8_t)nm_quant_i8(v[4 * i + 2], inv), b3 = (uint8_t)nm_quant_i8(v[4 * i + 3], inv);
+        w[i] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
     }
 }
 
-template <typename OutT> __device__ __forceinline__ void store1(OutT* p, float v, float) { *p = NmType<OutT>::from_f(v); }
-template <> __device__ __forceinline__ void store1<int8_t>(int8_t* p, float v, float inv) { *p = nm_quant_i8(v, inv); }
-
-template <typename OutT> __device__ __forceinline__ void add_res32(const uint4* p, float* v)
+// v[0..31] += 32 residual values held as packed words
+template <typename OutT> __device__ __forceinline__ void add_res32(const uint32_t* w, float* v);
+template <> __device__ __forceinline__ void add_res32<__nv_bfloat16>(const uint32_t* w, float* v)
 {
-    constexpr int PER = 16 / sizeof(OutT);
 #pragma unroll
-    for (int q = 0; q < 32 / PER; ++q) {
-        uint4 raw = p[q];
-        const OutT* e = reinterpret_cast<const OutT*>(&raw);
-#pragma unroll
-        for (int i = 0; i < PER; ++i) v[q * PER + i] += NmType<OutT>::to_f(e[i]);
+    for (int i = 0; i < 16; ++i) {
+        const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+        v[2 * i] += f.x;
+        v[2 * i + 1] += f.y;
     }
 }
-template <> __device__ __forceinline__ void add_res32<int8_t>(const uint4*, float*) {}
-template <typename OutT> __device__ __forceinline__ float res1(const OutT* p) { return NmType<OutT>::to_f(*p); }
-template <> __device__ __forceinline__ float res1<int8_t>(const int8_t*) { return 0.f; }
+template <> __device__ __forceinline__ void add_res32<__half>(const uint32_t* w, float* v)
+{
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        v[2 * i] += f.x;
+        v[2 * i + 1] += f.y;
+    }
+}
+template <> __device__ __forceinline__ void add_res32<float>(const uint32_t* w, float* v)
+{
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(w[i]);
+}
+template <> __device__ __forceinline__ void add_res32<int8_t>(const uint32_t*, float*) {}
 
-template <typename InT, typename OutT, int BN>
+template <typename InT, typename OutT, bool TWO>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const TcArgs a)
+linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                 const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmR, const TcArgs a)
 {
-    constexpr int B_BYTES = BN * ROW_BYTES;
+    constexpr int B_ROWS = TWO ? BN / 2 : BN;
+    constexpr int B_BYTES = B_ROWS * ROW_BYTES;
     constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    constexpr int TILE_M = TWO ? 2 * BM : BM;
     constexpr int BK_ELEMS = ROW_BYTES / (int)sizeof(InT);
-    constexpr uint32_t TMEM_COLS = 2 * BN;  // 512 or 256: a power of two
-    constexpr uint32_t IDESC = nm_idesc(TcIn<InT>::c_fmt, TcIn<InT>::ab_fmt, 0, 0, BM, BN);
+    constexpr uint32_t TMEM_COLS = 2 * BN;
+    constexpr uint32_t IDESC = nm_idesc(TcIn<InT>::c_fmt, TcIn<InT>::ab_fmt, 0, 0, TILE_M, BN);
+    // epilogue geometry: a warp owns 128 columns = 4 chunks of 32; a staging group is 128 bytes of
+    // output per row: 64 columns of a 16-bit type, 32 of fp32, 128 of int8
+    constexpr int NCH = BN / 64;
+    constexpr int GC = sizeof(OutT) == 4 ? 1 : (sizeof(OutT) == 2 ? 2 : 4);  // chunks per group
+    constexpr int NG = NCH / GC;                                             // groups per tile
+    constexpr int GROUP_COLS = 32 * GC;
+    constexpr int WPC = 32 / GC;  // packed words per chunk
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_full[MAX_STAGES];
     __shared__ uint64_t bar_empty[MAX_STAGES];
     __shared__ uint64_t bar_acc_full[2];
     __shared__ uint64_t bar_acc_empty[2];
+    __shared__ uint64_t bar_res[NUM_EPI_WARPS];
     __shared__ uint64_t bar_drain;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
+    const int stages = a.stages;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    float2* rep = reinterpret_cast<float2*>(tiles + (size_t)a.stages * STAGE_BYTES);
+    uint8_t* stage_out = tiles + (size_t)stages * STAGE_BYTES;   // 8 x 4 KB
+    uint8_t* stage_res = stage_out + NUM_EPI_WARPS * STAGE_BUF;   // 8 x 4 KB when a residual is given
+    float2* rep = reinterpret_cast<float2*>(stage_res + (a.has_res ? NUM_EPI_WARPS * STAGE_BUF : 0));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int stages = a.stages;
+    const uint32_t rank = TWO ? nm_cluster_ctarank() : 0u;  // 0 = leader of the pair
+    const int tile_first = TWO ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int tile_step = TWO ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
+        NM_TL(0);
         abort_flag = 0;
         nm_prefetch_tmap(&tmA);
         nm_prefetch_tmap(&tmW);
+        nm_prefetch_tmap(&tmO);
+        if (a.has_res) nm_prefetch_tmap(&tmR);
         for (int s = 0; s < stages; ++s) {
             nm_mbar_init(&bar_full[s], 1);
             nm_mbar_init(&bar_empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             nm_mbar_init(&bar_acc_full[b], 1);
-            nm_mbar_init(&bar_acc_empty[b], 8);
+            nm_mbar_init(&bar_acc_empty[b], TWO ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS);
         }
+        for (int w = 0; w < NUM_EPI_WARPS; ++w) nm_mbar_init(&bar_res[w], 1);
         nm_mbar_init(&bar_drain, 1);
         nm_fence_barrier_init();
     }
     if (warp == 1) {
-        nm_tmem_alloc(&tmem_slot, TMEM_COLS);
-        nm_tmem_relinquish();
+        if constexpr (TWO) {
+            nm_tmem_alloc2(&tmem_slot, TMEM_COLS);
+            nm_tmem_relinquish2();
+        } else {
+            nm_tmem_alloc(&tmem_slot, TMEM_COLS);
+            nm_tmem_relinquish();
+        }
     }
     if (a.tab) nm_table_replicate(rep, a.tab, a.n_seg, threadIdx.x, NUM_THREADS);
     nm_tc_fence_before();
     __syncthreads();
+    if constexpr (TWO) nm_cluster_sync();  // both CTAs' barriers and tensor memory are ready
     nm_tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_flag;
+    if (threadIdx.x == 0) NM_TL(1);
+    int tl_tile = 0;
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            long long issued = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
-                const int m0 = (tile / a.num_n_tiles) * BM;
-                const int n0 = (tile % a.num_n_tiles) * BN;
+            for (int tile = tile_first; ok && tile < a.num_tiles; tile += tile_step) {
+                const int m0 = (tile / a.num_n_tiles) * TILE_M + (int)rank * BM;
+                const int n0 = (tile % a.num_n_tiles) * BN + (int)rank * B_ROWS;
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
                     if (!nm_mbar_wait(&bar_empty[stage], phase ^ 1u, abortp, a.status)) { ok = false; break; }
+                    if (kb == 0 && tl_tile < 4) { NM_TL(4 + tl_tile); ++tl_tile; }
                     uint8_t* sa = tiles + (size_t)stage * STAGE_BYTES;
-                    nm_mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
-                    nm_tma_load_2d(sa, &tmA, kb * BK_ELEMS, m0, &bar_full[stage]);
-                    nm_tma_load_2d(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, &bar_full[stage]);
-                    ++issued;
+                    if constexpr (TWO) {
+                        // both CTAs' copies are counted on the leader's barrier
+                        const uint32_t full = nm_mapa(nm_smem_u32(&bar_full[stage]), 0);
+                        if (rank == 0) nm_mbar_expect_tx(&bar_full[stage], 2 * STAGE_BYTES);
+                        nm_tma_load_2d_2cta(sa, &tmA, kb * BK_ELEMS, m0, full);
+                        nm_tma_load_2d_2cta(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, full);
+                    } else {
+                        nm_mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
+                        nm_tma_load_2d(sa, &tmA, kb * BK_ELEMS, m0, &bar_full[stage]);
+                        nm_tma_load_2d(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, &bar_full[stage]);
+                    }
                     if (++stage == stages) { stage = 0; phase ^= 1u; }
                 }
             }
             if (!ok) {
-                // give the copies already issued a bounded time to land before the CTA retires
-                for (int s = 0; s < stages; ++s) {
-                    long long last = -1;  // last iteration that used stage s
-                    if (issued > s) last = ((issued - 1 - s) / stages) * stages + s;
-                    if (last < 0) continue;
-                    const uint32_t par = (uint32_t)((last / stages) & 1);
-                    long long t0 = clock64();
-                    while (!nm_mbar_try_wait(&bar_full[s], par) && clock64() - t0 < 200000000LL) {}
-                }
+                long long t0 = clock64();  // bounded pause: copies in flight land before teardown
+                while (clock64() - t0 < 4000000LL) {}
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------ MMA issuer (the leader CTA of a pair)
+        if (lane == 0 && rank == 0) {
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
-                if (!nm_mbar_wait(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status)) { ok = false; break; }
+            for (int tile = tile_first; ok && tile < a.num_tiles; tile += tile_step) {
+                if (!(TWO ? nm_mbar_wait_cluster(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status)
+                          : nm_mbar_wait(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status))) { ok = false; break; }
                 nm_tc_fence_after();
+                if (tl_tile < 4) NM_TL(8 + tl_tile);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
                     if (!nm_mbar_wait(&bar_full[stage], phase, abortp, a.status)) { ok = false; break; }
+                    if (kb == 0 && tl_tile < 4) NM_TL(12 + tl_tile);
                     nm_tc_fence_after();
                     const uint32_t sa = nm_smem_u32(tiles + (size_t)stage * STAGE_BYTES);
                     const uint64_t adesc = nm_smem_desc_sw128(sa);
@@ -218,164 +276,211 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {  // 4 x 32 bytes of K per 128-byte row
                         const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-                        if constexpr (TcIn<InT>::is_int) nm_mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
-                        else nm_mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                        if constexpr (TWO) {
+                            if constexpr (TcIn<InT>::is_int) nm_mma_i8_2cta(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                            else nm_mma_f16_2cta(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                        } else {
+                            if constexpr (TcIn<InT>::is_int) nm_mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                            else nm_mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                        }
                     }
-                    nm_tc_commit(&bar_empty[stage]);  // smem stage reusable once these MMAs retire
+                    // smem stage reusable (in both CTAs of a pair) once these MMAs retire
+                    if constexpr (TWO) nm_tc_commit2(&bar_empty[stage], 3);
+                    else nm_tc_commit(&bar_empty[stage]);
                     if (++stage == stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                nm_tc_commit(&bar_acc_full[buf]);
+                if constexpr (TWO) nm_tc_commit2(&bar_acc_full[buf], 3);
+                else nm_tc_commit(&bar_acc_full[buf]);
+                if (tl_tile < 4) { NM_TL(16 + tl_tile); ++tl_tile; }
                 buf ^= 1;
                 if (buf == 0) acc_phase ^= 1u;
             }
             if (!ok) {
-                nm_tc_commit(&bar_drain);
+                if constexpr (TWO) nm_tc_commit2(&bar_drain, 1);
+                else nm_tc_commit(&bar_drain);
                 long long t0 = clock64();
                 while (!nm_mbar_try_wait(&bar_drain, 0) && clock64() - t0 < 200000000LL) {}
             }
         }
     } else {
         // ------------------------------------------------ epilogue (warps 2..9)
-        // Two warps per tensor-memory lane quarter; each takes half of the tile's columns in
-        // 32-column chunks.  The tensor-memory load and the residual load of chunk i+1 are in
-        // flight while chunk i is computed and stored.
-        const int q = warp & 3;              // lane quarter this warp may read
-        const int half = (warp - 2) >> 2;    // which half of the columns
-        constexpr int NCH = BN / 64;         // chunks per warp per tile
-        constexpr int RV = 2 * (int)sizeof(OutT);  // 16-byte vectors of residual per 32 columns
+        const int e = warp - 2;   // epilogue warp index
+        const int q = warp & 3;   // tensor-memory lane quarter this warp may read
+        const int half = e >> 2;  // which half of the tile's columns
+        uint8_t* my_out = stage_out + e * STAGE_BUF;
+        uint8_t* my_res = stage_res + e * STAGE_BUF;
+        const uint32_t my_out_row = nm_smem_u32(my_out) + (uint32_t)lane * 128u;
+        const uint32_t my_res_row = nm_smem_u32(my_res) + (uint32_t)lane * 128u;
+        const uint32_t rep_lane = nm_smem_u32(rep) + (uint32_t)lane * 8u;
         int buf = 0;
         uint32_t acc_phase = 0;
+        uint32_t res_phase = 0;
         const bool has_tab = a.tab != nullptr;
+        const bool has_res = a.has_res != 0;
         const float inv_h = has_tab ? a.tab->inv_h : 0.f;
         const float off = has_tab ? a.tab->off : 0.f;
         const float nm1 = (float)(a.n_seg - 1);
-        OutT* out = reinterpret_cast<OutT*>(a.out);
-        const OutT* res = reinterpret_cast<const OutT*>(a.residual);
-        for (int tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x) {
-            const int m0 = (tile / a.num_n_tiles) * BM;
+        // residual of the first group of the first tile
+        if (has_res && lane == 0 && tile_first < a.num_tiles) {
+            const int m0 = (tile_first / a.num_n_tiles) * TILE_M + (int)rank * BM;
+            const int n0 = (tile_first % a.num_n_tiles) * BN + half * (BN / 2);
+            nm_mbar_expect_tx(&bar_res[e], STAGE_BUF);
+            nm_tma_load_2d(my_res, &tmR, n0, m0 + q * 32, &bar_res[e]);
+        }
+        int ok = 1;
+        for (int tile = tile_first; ok && tile < a.num_tiles; tile += tile_step) {
+            const int m0 = (tile / a.num_n_tiles) * TILE_M + (int)rank * BM;
             const int n0 = (tile % a.num_n_tiles) * BN + half * (BN / 2);
-            int ok = 1;
             if (lane == 0) ok = nm_mbar_wait(&bar_acc_full[buf], acc_phase, abortp, a.status) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
+            (void)nm_mbar_try_wait(&bar_acc_full[buf], acc_phase);  // every lane observes the phase itself
             nm_tc_fence_after();
+            if (warp == 2 && lane == 0 && tl_tile < 4) NM_TL(20 + tl_tile);
             const int64_t row = (int64_t)m0 + q * 32 + lane;
             const bool row_ok = row < a.M;
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2));
             uint32_t r[2][32];
-            uint4 rs[2][RV];
             nm_tmem_ld32_async(t_addr, r[0]);
-            if (res && row_ok && n0 + 32 <= a.N) {
 #pragma unroll
-                for (int v = 0; v < RV; ++v) rs[0][v] = __ldg(reinterpret_cast<const uint4*>(res + row * a.ldr + n0) + v);
-            }
+            for (int g = 0; g < NG; ++g) {
+                uint32_t packed[32];
+                uint32_t rsv[32];
+                if (has_res) {
+                    if (lane == 0) ok = nm_mbar_wait(&bar_res[e], res_phase, abortp, a.status) ? 1 : 0;
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (ok) (void)nm_mbar_try_wait(&bar_res[e], res_phase);  // every lane observes the phase itself
+                    res_phase ^= 1u;
 #pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                const int cur = c & 1;
-                nm_tmem_ld_wait32(r[cur]);
-                const int64_t col0 = (int64_t)n0 + c * 32;
-                if (c + 1 < NCH) {
-                    nm_tmem_ld32_async(t_addr + (uint32_t)((c + 1) * 32), r[cur ^ 1]);
-                    if (res && row_ok && col0 + 64 <= a.N) {
-#pragma unroll
-                        for (int v = 0; v < RV; ++v)
-                            rs[cur ^ 1][v] = __ldg(reinterpret_cast<const uint4*>(res + row * a.ldr + col0 + 32) + v);
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t addr = my_res_row + (uint32_t)((c ^ (lane & 7)) << 4);
+                        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(rsv[4 * c]), "=r"(rsv[4 * c + 1]), "=r"(rsv[4 * c + 2]), "=r"(rsv[4 * c + 3])
+                                     : "r"(addr));
                     }
-                } else {
-                    // this warp's share of the accumulator is in registers: hand the buffer back
-                    nm_tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) nm_mbar_arrive(&bar_acc_empty[buf]);
-                    __syncwarp();
+                    // the buffer is free again: fetch the residual of the next group (this tile's, or
+                    // the first group of this CTA's next tile) while this one is computed
+                    if (lane == 0 && ok) {
+                        int nm0 = m0, nn0 = n0 + (g + 1) * GROUP_COLS;
+                        bool more = true;
+                        if (g + 1 == NG) {
+                            const int nt = tile + tile_step;
+                            more = nt < a.num_tiles;
+                            nm0 = (nt / a.num_n_tiles) * TILE_M + (int)rank * BM;
+                            nn0 = (nt % a.num_n_tiles) * BN + half * (BN / 2);
+                        }
+                        if (more) {
+                            nm_mbar_expect_tx(&bar_res[e], STAGE_BUF);
+                            nm_tma_load_2d(my_res, &tmR, nn0, nm0 + q * 32, &bar_res[e]);
+                        }
+                    }
                 }
-                // lanes beyond the last row / column skip the arithmetic but stay in the loop:
-                // the tensor-memory loads need the whole warp
-                if (row_ok && col0 < a.N) {
-                    float v[32];
-                    if (col0 + 32 <= a.N) {
-                        if constexpr (TcIn<InT>::is_int) {
-                            if (a.acc_dump) {
 #pragma unroll
-                                for (int i = 0; i < 32; i += 4)
+                for (int cc = 0; cc < GC; ++cc) {
+                    const int c = g * GC + cc;
+                    const int cur = c & 1;
+                    nm_tmem_ld_wait32(r[cur]);
+                    if (c + 1 < NCH) {
+                        nm_tmem_ld32_async(t_addr + (uint32_t)((c + 1) * 32), r[cur ^ 1]);
+                    } else {
+                        // this warp's share of the accumulator is in registers: hand the buffer back
+                        nm_tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if constexpr (TWO) nm_mbar_arrive_cluster(nm_mapa(nm_smem_u32(&bar_acc_empty[buf]), 0));
+                            else nm_mbar_arrive(&bar_acc_empty[buf]);
+                        }
+                        __syncwarp();
+                    }
+                    const int64_t col0 = (int64_t)n0 + c * 32;
+                    float v[32];
+                    // columns beyond N are computed on zero operands and clipped by the TMA store;
+                    // only the loads of bias / scale and the debug dumps need the bound
+                    if constexpr (TcIn<InT>::is_int) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            float4 ws = make_float4(0.f, 0.f, 0.f, 0.f), bs = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (col0 + i < a.N) {
+                                ws = __ldg(reinterpret_cast<const float4*>(a.w_scale + col0 + i));
+                                if (a.bias) bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
+                                if (a.acc_dump && row_ok)
                                     *reinterpret_cast<int4*>(a.acc_dump + row * a.N + col0 + i) =
                                         make_int4((int)r[cur][i], (int)r[cur][i + 1], (int)r[cur][i + 2], (int)r[cur][i + 3]);
                             }
+                            v[i] = __fmaf_rn((float)(int)r[cur][i], a.a_scale * ws.x, bs.x);
+                            v[i + 1] = __fmaf_rn((float)(int)r[cur][i + 1], a.a_scale * ws.y, bs.y);
+                            v[i + 2] = __fmaf_rn((float)(int)r[cur][i + 2], a.a_scale * ws.z, bs.z);
+                            v[i + 3] = __fmaf_rn((float)(int)r[cur][i + 3], a.a_scale * ws.w, bs.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[cur][i]);
+                        if (a.bias) {
 #pragma unroll
                             for (int i = 0; i < 32; i += 4) {
-                                const float4 ws = __ldg(reinterpret_cast<const float4*>(a.w_scale + col0 + i));
-                                float4 bs = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (a.bias) bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
-                                v[i] = __fmaf_rn((float)(int)r[cur][i], a.a_scale * ws.x, bs.x);
-                                v[i + 1] = __fmaf_rn((float)(int)r[cur][i + 1], a.a_scale * ws.y, bs.y);
-                                v[i + 2] = __fmaf_rn((float)(int)r[cur][i + 2], a.a_scale * ws.z, bs.z);
-                                v[i + 3] = __fmaf_rn((float)(int)r[cur][i + 3], a.a_scale * ws.w, bs.w);
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[cur][i]);
-                            if (a.bias) {
-#pragma unroll
-                                for (int i = 0; i < 32; i += 4) {
+                                if (col0 + i < a.N) {
                                     const float4 bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
                                     v[i] += bs.x; v[i + 1] += bs.y; v[i + 2] += bs.z; v[i + 3] += bs.w;
                                 }
                             }
                         }
-                        if (has_tab) {
-                            if (a.idx_dump) {
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) {
-                                    int s;
-                                    v[i] = nm_pwl_eval_rep(rep, lane, v[i], inv_h, off, nm1, &s);
-                                    a.idx_dump[row * a.N + col0 + i] = s;
-                                }
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) v[i] = nm_pwl_eval_rep(rep, lane, v[i], inv_h, off, nm1);
-                            }
-                        }
-                        if (res) add_res32<OutT>(rs[cur], v);
-                        store32<OutT>(out + row * a.ldo + col0, v, a.inv_out_scale);
-                    } else {
-                        // ragged right edge: element by element
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int64_t col = col0 + i;
-                            if (col >= a.N) continue;
-                            float x;
-                            const float bj = a.bias ? a.bias[col] : 0.f;
-                            if constexpr (TcIn<InT>::is_int) {
-                                if (a.acc_dump) a.acc_dump[row * a.N + col] = (int)r[cur][i];
-                                x = __fmaf_rn((float)(int)r[cur][i], a.a_scale * a.w_scale[col], bj);
-                            } else {
-                                x = __uint_as_float(r[cur][i]) + bj;
-                            }
-                            if (has_tab) {
-                                int s;
-                                x = nm_pwl_eval_rep(rep, lane, x, inv_h, off, nm1, &s);
-                                if (a.idx_dump) a.idx_dump[row * a.N + col] = s;
-                            }
-                            if (res) x += res1<OutT>(res + row * a.ldr + col);
-                            store1<OutT>(out + row * a.ldo + col, x, a.inv_out_scale);
-                        }
                     }
+                    if (has_tab) {
+                        if (a.idx_dump) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                int s;
+                                v[i] = nm_pwl_fast(rep_lane, v[i], inv_h, off, nm1, &s);
+                                if (row_ok && col0 + i < a.N) a.idx_dump[row * a.N + col0 + i] = s;
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = nm_pwl_fast(rep_lane, v[i], inv_h, off, nm1);
+                        }
+                    } else if (a.idx_dump) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (row_ok && col0 + i < a.N) a.idx_dump[row * a.N + col0 + i] = -1;
+                    }
+                    if (has_res) add_res32<OutT>(&rsv[cc * WPC], v);
+                    pack32<OutT>(v, &packed[cc * WPC], a.inv_out_scale);
                 }
+                // stage the group and send it: the previous store must have finished reading the buffer
+                if (lane == 0) nm_tma_store_wait_read();
                 __syncwarp();
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t addr = my_out_row + (uint32_t)((c ^ (lane & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(packed[4 * c]),
+                                 "r"(packed[4 * c + 1]), "r"(packed[4 * c + 2]), "r"(packed[4 * c + 3])
+                                 : "memory");
+                }
+                nm_fence_proxy_async();
+                __syncwarp();
+                // a group that lies wholly beyond the matrix is not stored at all
+                if (lane == 0 && ok && n0 + g * GROUP_COLS < a.N && m0 + q * 32 < a.M)
+                    nm_tma_store_2d(&tmO, my_out, n0 + g * GROUP_COLS, m0 + q * 32);
             }
+            if (warp == 2 && lane == 0 && tl_tile < 4) { NM_TL(24 + tl_tile); ++tl_tile; }
             buf ^= 1;
             if (buf == 0) acc_phase ^= 1u;
         }
+        if (lane == 0) nm_tma_store_wait_read();  // staging memory must outlive the last store's reads
+        __syncwarp();
     }
-
 
     // ---------------------------------------------------- teardown (all paths)
     nm_tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) NM_TL(2);
+    if constexpr (TWO) nm_cluster_sync();  // the peer may still use barriers / tensor memory of the pair
     if (warp == 1) {
         __syncwarp();
         nm_tc_fence_after();
-        nm_tmem_dealloc(tmem_base, TMEM_COLS);
+        if constexpr (TWO) nm_tmem_dealloc2(tmem_base, TMEM_COLS);
+        else nm_tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -383,13 +488,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 2-D K-contiguous matrix [rows, cols] with row pitch ld (elements); box = 128 bytes x box_rows.
+// 2-D row-major matrix [rows, cols] with row pitch ld (elements); box = 128 bytes x box_rows, 128-byte swizzle.
 nm_status make_tmap(nm_ctx* ctx, CUtensorMap* m, const void* base, nm_dtype dt, int64_t rows, int64_t cols,
                     int64_t ld, int box_rows)
 {
     const size_t es = nm_dtype_size(dt);
-    CUtensorMapDataType t = dt == NM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+    CUtensorMapDataType t = dt == NM_BF16  ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
                             : dt == NM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                            : dt == NM_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                            : CU_TENSOR_MAP_DATA_TYPE_UINT8;
     cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t gstr[1] = {(cuuint64_t)ld * es};
@@ -402,52 +508,93 @@ nm_status make_tmap(nm_ctx* ctx, CUtensorMap* m, const void* base, nm_dtype dt, 
     return r == CUDA_SUCCESS ? NM_OK : NM_ERR_CUDA;
 }
 
-template <typename InT, typename OutT, int BN>
+template <typename InT, typename OutT, bool TWO>
 nm_status launch(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
 {
-    constexpr int STAGE_BYTES = A_BYTES + BN * ROW_BYTES;
+    constexpr int B_ROWS = TWO ? BN / 2 : BN;
+    constexpr int TILE_M = TWO ? 2 * BM : BM;
+    constexpr int STAGE_BYTES = A_BYTES + B_ROWS * ROW_BYTES;
     TcArgs a;
-    a.M = d->M; a.N = d->N; a.K = d->K; a.ldr = d->ldr; a.ldo = d->ldo;
-    a.bias = d->bias; a.residual = d->residual; a.out = d->out;
+    memset(&a, 0, sizeof(a));
+    a.M = d->M; a.N = d->N; a.K = d->K;
+    a.bias = d->bias;
+    a.has_res = d->residual ? 1 : 0;
     a.tab = d->slot == NM_SLOT_NONE ? nullptr : ctx->d_tables + d->slot;
     a.n_seg = d->slot == NM_SLOT_NONE ? 0 : ctx->h_tables[d->slot].n;
     a.a_scale = d->a_scale; a.w_scale = d->w_scale; a.inv_out_scale = d->inv_out_scale;
     a.acc_dump = d->acc_dump; a.idx_dump = d->idx_dump;
     a.status = ctx->d_status;
+#ifdef NM_EXP_TIMELINE
+    a.dbg = getenv("NM_DBG_PTR") ? (long long*)strtoull(getenv("NM_DBG_PTR"), nullptr, 16) : nullptr;
+#endif
     const int bk = ROW_BYTES / (int)sizeof(InT);
-    const int64_t m_tiles = (d->M + BM - 1) / BM;
+    const int64_t m_tiles = (d->M + TILE_M - 1) / TILE_M;
     a.num_n_tiles = (int)((d->N + BN - 1) / BN);
     if (m_tiles * a.num_n_tiles > 0x7fffffffLL) return NM_ERR_SHAPE;
     a.num_tiles = (int)(m_tiles * a.num_n_tiles);
     a.num_k_blocks = (int)((d->K + bk - 1) / bk);
     const size_t table_bytes = (size_t)a.n_seg * 32 * sizeof(float2);
-    const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - table_bytes;
+    const size_t staging = (size_t)NUM_EPI_WARPS * STAGE_BUF * (a.has_res ? 2 : 1);
+    const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - table_bytes - staging;
     int stages = (int)(budget / STAGE_BYTES);
     if (stages > MAX_STAGES) stages = MAX_STAGES;
     if (stages < 2) return NM_ERR_UNSUPPORTED;
     a.stages = stages;
-    const size_t smem = (size_t)stages * STAGE_BYTES + table_bytes + 1024;
+    const size_t smem = (size_t)stages * STAGE_BYTES + staging + table_bytes + 1024;
 
-    CUtensorMap tmA, tmW;
+    CUtensorMap tmA, tmW, tmO, tmR;
     nm_status s = make_tmap(ctx, &tmA, d->A, d->in_dtype, d->M, d->K, d->lda, BM);
     if (s != NM_OK) return s;
-    s = make_tmap(ctx, &tmW, d->W, d->in_dtype, d->N, d->K, d->ldw, BN);
+    s = make_tmap(ctx, &tmW, d->W, d->in_dtype, d->N, d->K, d->ldw, B_ROWS);
+    if (s != NM_OK) return s;
+    s = make_tmap(ctx, &tmO, d->out, d->out_dtype, d->M, d->N, d->ldo, 32);
+    if (s != NM_OK) return s;
+    if (d->residual) s = make_tmap(ctx, &tmR, d->residual, d->out_dtype, d->M, d->N, d->ldr, 32);
+    else tmR = tmO;
     if (s != NM_OK) return s;
 
-    auto kern = linear_tc_kernel<InT, OutT, BN>;
+    auto kern = linear_tc_kernel<InT, OutT, TWO>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return NM_ERR_CUDA;
-    const int grid = a.num_tiles < ctx->sm_count ? a.num_tiles : ctx->sm_count;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if constexpr (TWO) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        // persistent: no more clusters than can be resident at once (cached per kernel and smem size)
+        static int max_clusters = 0;
+        static size_t max_clusters_smem = 0;
+        if (max_clusters == 0 || max_clusters_smem != smem) {
+            cfg.gridDim = dim3(2 * (unsigned)(ctx->sm_count / 2));
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) return NM_ERR_CUDA;
+            max_clusters = n;
+            max_clusters_smem = smem;
+        }
+        const int pairs = a.num_tiles < max_clusters ? a.num_tiles : max_clusters;
+        cfg.gridDim = dim3(2 * (unsigned)pairs);
+    } else {
+        cfg.gridDim = dim3((unsigned)(a.num_tiles < ctx->sm_count ? a.num_tiles : ctx->sm_count));
+    }
     NmLaunchScope scope(ctx, NM_KERNEL_LINEAR_TC, 2.0 * (double)d->M * (double)d->N * (double)d->K, st);
-    kern<<<grid, NUM_THREADS, smem, st>>>(tmA, tmW, a);
+    if (cudaLaunchKernelEx(&cfg, kern, tmA, tmW, tmO, tmR, a) != cudaSuccess) return NM_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
 }
 
 template <typename InT, typename OutT>
-nm_status launch_bn(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
+nm_status launch_sel(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
 {
-    if (d->N % 256 == 0 || d->N >= 1024) return launch<InT, OutT, 256>(ctx, d, st);
-    return launch<InT, OutT, 128>(ctx, d, st);
+    // algo 3 forces the one-CTA tile; otherwise problems with at least one 256 x 256 tile use CTA pairs
+    if (d->algo != 3 && d->M >= 256 && d->N >= 256) return launch<InT, OutT, true>(ctx, d, st);
+    return launch<InT, OutT, false>(ctx, d, st);
 }
 
 }  // namespace
@@ -458,7 +605,7 @@ bool nm_linear_tc_supported(const nm_linear_desc* d)
     const size_t es = nm_dtype_size(d->in_dtype);
     if (d->M < 1 || d->N < 8 || d->K < 1) return false;
     if ((d->K * es) % 16 != 0) return false;  // TMA: global extents and pitches in 16-byte units
-    if (d->N % 4 != 0) return false;          // vector dumps / bias loads
+    if (d->N % 4 != 0) return false;          // vector loads of bias / scales, vector dumps
     if (d->in_dtype == NM_I8) return d->out_dtype == NM_BF16 || d->out_dtype == NM_F32 || d->out_dtype == NM_I8;
     return d->out_dtype == d->in_dtype;
 }
@@ -467,12 +614,12 @@ nm_status nm_launch_linear_tc(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t
 {
     if (!nm_linear_tc_supported(d)) return NM_ERR_UNSUPPORTED;
     switch (d->in_dtype) {
-    case NM_BF16: return launch_bn<__nv_bfloat16, __nv_bfloat16>(ctx, d, st);
-    case NM_F16: return launch_bn<__half, __half>(ctx, d, st);
+    case NM_BF16: return launch_sel<__nv_bfloat16, __nv_bfloat16>(ctx, d, st);
+    case NM_F16: return launch_sel<__half, __half>(ctx, d, st);
     case NM_I8:
-        if (d->out_dtype == NM_BF16) return launch_bn<int8_t, __nv_bfloat16>(ctx, d, st);
-        if (d->out_dtype == NM_F32) return launch_bn<int8_t, float>(ctx, d, st);
-        return launch_bn<int8_t, int8_t>(ctx, d, st);
+        if (d->out_dtype == NM_BF16) return launch_sel<int8_t, __nv_bfloat16>(ctx, d, st);
+        if (d->out_dtype == NM_F32) return launch_sel<int8_t, float>(ctx, d, st);
+        return launch_sel<int8_t, int8_t>(ctx, d, st);
     default: return NM_ERR_UNSUPPORTED;
     }
 }

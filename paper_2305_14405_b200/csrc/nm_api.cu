@@ -234,7 +234,7 @@ nm_status nm_linear_pwl(nm_ctx* ctx, const nm_linear_desc* d, void* stream)
     cudaStream_t st = (cudaStream_t)stream;
     if (d->algo == 1) return nm_launch_linear_simt(ctx, d, st);
     const bool tc = nm_linear_tc_supported(d);
-    if (d->algo == 2) return tc ? nm_launch_linear_tc(ctx, d, st) : NM_ERR_UNSUPPORTED;
+    if (d->algo == 2 || d->algo == 3) return tc ? nm_launch_linear_tc(ctx, d, st) : NM_ERR_UNSUPPORTED;
     // tiny problems do not fill a 128-row tensor-core tile; the CUDA-core kernel takes them
     if (tc && d->M >= 64 && d->N >= 64) return nm_launch_linear_tc(ctx, d, st);
     return nm_launch_linear_simt(ctx, d, st);

@@ -212,6 +212,41 @@ __device__ __forceinline__ void nm_tma_load_3d(void* smem_dst, const CUtensorMap
         : "memory");
 }
 
+// TMA: 2-D tiled store shared -> global as one bulk group; parts of the box beyond the
+// tensor's extents are not written.  c0 (innermost) must be a multiple of 16 bytes.
+__device__ __forceinline__ void nm_tma_store_2d(const CUtensorMap* tmap, const void* smem_src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tmap),
+                 "r"(nm_smem_u32(smem_src)), "r"(c0), "r"(c1)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// All earlier bulk stores of this thread have finished READING shared memory (the
+// staging buffer may be overwritten; the global writes may still be in flight).
+__device__ __forceinline__ void nm_tma_store_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
+// PWL lookup for hot loops.  `rep_lane` is the shared::cta byte address of this lane's
+// column of a 32-way replicated table (entry s of lane l at rep + (s*32 + l)*8).  The segment
+// number is floor(clamp(fma(x, inv_h, off), 0, n-1)): the floor is taken by adding 1.5*2^23
+// with round-toward-minus-infinity, which leaves floor(u) in the low mantissa bits (exact for
+// 0 <= u < 2^22), and the table address is formed from those bits with one shift-add.
+__device__ __forceinline__ float nm_pwl_fast(uint32_t rep_lane, float x, float inv_h, float off, float nm1,
+                                             int* idx_out = nullptr)
+{
+    float u = __fmaf_rn(x, inv_h, off);
+    u = fminf(fmaxf(u, 0.0f), nm1);
+    const uint32_t bits = __float_as_uint(__fadd_rd(u, 12582912.0f));   // 0x4B400000 + floor(u)
+    if (idx_out) *idx_out = (int)(bits - 0x4B400000u);
+    // (bits << 8) = 0x40000000 + s*256 (mod 2^32); the constant is folded into the base
+    const uint32_t addr = (bits << 8) + (rep_lane - 0x40000000u);
+    float k, b;
+    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(k), "=f"(b) : "r"(addr));   // the table is read-only here
+    return __fmaf_rn(k, x, b);
+}
+
 __device__ __forceinline__ void nm_prefetch_tmap(const CUtensorMap* tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
@@ -266,6 +301,116 @@ __device__ __forceinline__ void nm_mma_i8(uint32_t d_tmem, uint64_t adesc, uint6
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// ---- thread-block clusters and two-CTA tensor-core groups (cta_group::2) ----------
+
+__device__ __forceinline__ uint32_t nm_cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the object at shared::cta address `addr` in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t nm_mapa(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void nm_mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void nm_cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ bool nm_mbar_try_wait_cluster(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(nm_smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait, cluster-scope acquire (the arrivals come from the peer CTA as well).
+__device__ __forceinline__ bool nm_mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                     int* status)
+{
+    if (nm_mbar_try_wait_cluster(bar, parity)) return true;
+    long long t0 = clock64();
+    uint32_t spins = 0;
+    while (true) {
+        if (nm_mbar_try_wait_cluster(bar, parity)) return true;
+        if ((++spins & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > NM_WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, (int)NM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+// TMA load whose completion is counted on an mbarrier that may live in the peer CTA of a
+// two-CTA group (`bar_cluster_addr` is a shared::cluster address).  Each CTA fetches its own
+// operand slice into its own shared memory.
+__device__ __forceinline__ void nm_tma_load_2d_2cta(void* smem_dst, const CUtensorMap* tmap, int c0, int c1,
+                                                    uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(nm_smem_u32(smem_dst)), "l"(tmap), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void nm_tmem_alloc2(uint32_t* smem_slot, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(nm_smem_u32(smem_slot)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void nm_tmem_relinquish2()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void nm_tmem_dealloc2(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// Commit of a two-CTA group: arrives once on the barrier at the same shared-memory offset
+// in every CTA named by `cta_mask`.
+__device__ __forceinline__ void nm_tc_commit2(uint64_t* bar, uint16_t cta_mask)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+            nm_smem_u32(bar)),
+        "h"(cta_mask)
+        : "memory");
+}
+// One MMA over both CTAs of the pair: M = 256 (128 rows of A and of D per CTA), B split
+// along N between the two CTAs' shared memories.  Issued by the leader CTA only.
+__device__ __forceinline__ void nm_mma_f16_2cta(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void nm_mma_i8_2cta(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }

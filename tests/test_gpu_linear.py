@@ -48,20 +48,25 @@ def test_linear_f32_simt(nm, ctx, M, N, K, epi):
     assert_close_f32(got, ref, "linear f32 %s" % epi)
 
 
+@pytest.mark.parametrize("algo", ["tc", "tc_1cta"])
 @pytest.mark.parametrize("dtype", ["bf16", "f16"])
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 256, 128), (384, 768, 768), (128, 128, 256),
-                                   (200, 328, 72), (130, 136, 1032), (1024, 2304, 768)])
-def test_linear_tc_plain(nm, ctx, dtype, M, N, K):
-    """Several tiles, ragged rows / columns / K, both tile widths."""
-    got, ref = run_float(nm, ctx, dtype, M, N, K, False, False, None, nm.ALGO_TC)
-    assert_close_bf16(got, ref, "linear tc %s %dx%dx%d" % (dtype, M, N, K))
+                                   (200, 328, 72), (130, 136, 1032), (1024, 2304, 768), (600, 520, 200)])
+def test_linear_tc_plain(nm, ctx, algo, dtype, M, N, K):
+    """Several tiles, ragged rows / columns / K, both tile widths; "tc" uses CTA pairs
+    (cta_group::2, 256-row tiles) once M and N reach 256, "tc_1cta" forces one CTA per tile."""
+    a = nm.ALGO_TC if algo == "tc" else nm.ALGO_TC_1CTA
+    got, ref = run_float(nm, ctx, dtype, M, N, K, False, False, None, a)
+    assert_close_bf16(got, ref, "linear %s %s %dx%dx%d" % (algo, dtype, M, N, K))
 
 
+@pytest.mark.parametrize("algo", ["tc", "tc_1cta"])
 @pytest.mark.parametrize("epi", ["gelu_bias", "bias_res", "relu_bias_res"])
-@pytest.mark.parametrize("M,N,K", [(256, 512, 192), (200, 328, 72), (512, 3072, 768)])
-def test_linear_tc_epilogues(nm, ctx, epi, M, N, K):
+@pytest.mark.parametrize("M,N,K", [(256, 512, 192), (200, 328, 72), (512, 3072, 768), (700, 776, 136)])
+def test_linear_tc_epilogues(nm, ctx, algo, epi, M, N, K):
     slot = "gelu" if epi == "gelu_bias" else ("relu" if epi == "relu_bias_res" else None)
-    got, ref = run_float(nm, ctx, "bf16", M, N, K, True, "res" in epi, slot, nm.ALGO_TC, seed=5)
+    a = nm.ALGO_TC if algo == "tc" else nm.ALGO_TC_1CTA
+    got, ref = run_float(nm, ctx, "bf16", M, N, K, True, "res" in epi, slot, a, seed=5)
     assert_close_bf16(got, ref, "linear tc %s" % epi)
 
 
@@ -72,9 +77,9 @@ def test_linear_tc_matches_simt_path_choice(nm, ctx):
         assert_close_bf16(got, ref, "algo %d" % algo)
 
 
-@pytest.mark.parametrize("algo", ["simt", "tc"])
+@pytest.mark.parametrize("algo", ["simt", "tc", "tc_1cta"])
 @pytest.mark.parametrize("M,N,K,out", [(256, 256, 256, "bf16"), (200, 328, 144, "bf16"), (384, 1024, 1024, "i8"),
-                                       (128, 512, 4096, "f32")])
+                                       (128, 512, 4096, "f32"), (512, 512, 512, "f32")])
 def test_linear_int8_bit_exact(nm, ctx, algo, M, N, K, out):
     """int32 accumulators and segment numbers must match the oracle bit for bit; so must the
     fp32 epilogue value and the requantised int8 output."""
@@ -94,7 +99,7 @@ def test_linear_int8_bit_exact(nm, ctx, algo, M, N, K, out):
     idx = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
     ctx.linear_pwl(Ad, Wd, o, bias=torch.from_numpy(bias).cuda(), slot=nm.SLOT_GELU, a_scale=float(a_scale),
                    w_scale=torch.from_numpy(ws).cuda(), inv_out_scale=inv, acc_dump=acc, idx_dump=idx,
-                   algo=nm.ALGO_SIMT if algo == "simt" else nm.ALGO_TC)
+                   algo={"simt": nm.ALGO_SIMT, "tc": nm.ALGO_TC, "tc_1cta": nm.ALGO_TC_1CTA}[algo])
     ctx.check_device_status()
     r = oracle.linear_i8(Aq, Wq, a_scale, ws, bias, None, tabs["gelu"], out_scale=out_scale)
     assert np.array_equal(acc.cpu().numpy(), r["acc"])
