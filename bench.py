@@ -26,6 +26,9 @@ if ROOT not in sys.path:
 METRIC = "PWL BERT encoder tokens/s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, mean over the four
+# GEMM shapes of a layer, from the ncu capture summarised in profiles/encoder_c3_launches_and_kernels.md
+NCU_GEMM_DRAM_BYTES_PER_LAUNCH = {"c3_bert_base_12l_bf16": 80.5e6}
 
 
 def parse_args():
@@ -296,7 +299,8 @@ def main():
         achieved = work_l / (ms_l * 1e-3) / 1e12 if ms_l > 0 else 0.0
         peak = peaks["bf16_tflops_sustained"] if cfg.dtype != "f32" else peaks["bf16_tflops_sustained"] / 2
         roofline = {"bound": "tensor", "kernel": gemm_kind, "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name),
                     "peak_source": "%s (bf16 sustained: kernel timed inside a long step)" % peak_kind,
                     "avg_launch_us": ms_l / max(n_l, 1) * 1e3, "share_of_step": ms_l / total_ms}
         extra = {}
@@ -326,12 +330,16 @@ def main():
             "whole_step_tflops": whole,
         }
         if not args.no_cpu_baseline and world == 1:
-            n_layers = cfg.layers if cfg.T * cfg.H * cfg.layers <= 512 * 768 * 12 else max(1, cfg.layers // 4)
-            v, secs, cores = time_oracle(cfg, x_np, layers_np, min(n_layers, cfg.layers), 1)
+            # calibrate on one sequence through one layer, then size the sample to ~15 s of CPU work
+            _, t1, _ = time_oracle(cfg, x_np, layers_np, 1, 1)
+            n_layers = max(1, min(cfg.layers, int(15.0 / max(t1, 1e-3))))
+            n_seq = max(1, min(cfg.B, int(15.0 / max(t1 * n_layers, 1e-3))))
+            v, secs, cores = time_oracle(cfg, x_np, layers_np, n_layers, n_seq)
             line["cpu_baseline"] = {
                 "value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                "sample": "1 of %d sequences (%d tokens) through %d of %d layers, %.1f s; scaled by layers"
-                          % (cfg.B, cfg.L, min(n_layers, cfg.layers), cfg.layers, secs)}
+                "sample": "%d of %d sequences (%d tokens each) through %d of %d layers, %.1f s%s"
+                          % (n_seq, cfg.B, cfg.L, n_layers, cfg.layers, secs,
+                             "" if n_layers == cfg.layers else "; scaled by the layer count")}
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

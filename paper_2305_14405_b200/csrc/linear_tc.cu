@@ -332,7 +332,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int tile = tile_first; ok && tile < a.num_tiles; tile += tile_step) {
             const int m0 = (tile / a.num_n_tiles) * TILE_M + (int)rank * BM;
             const int n0 = (tile % a.num_n_tiles) * BN + half * (BN / 2);
-            if (lane == 0) ok = nm_mbar_wait(&bar_acc_full[buf], acc_phase, abortp, a.status) ? 1 : 0;
+            if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_acc_full[buf], acc_phase, abortp, a.status) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             (void)nm_mbar_try_wait(&bar_acc_full[buf], acc_phase);  // every lane observes the phase itself
@@ -348,7 +348,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 uint32_t packed[32];
                 uint32_t rsv[32];
                 if (has_res) {
-                    if (lane == 0) ok = nm_mbar_wait(&bar_res[e], res_phase, abortp, a.status) ? 1 : 0;
+                    if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_res[e], res_phase, abortp, a.status) ? 1 : 0;
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (ok) (void)nm_mbar_try_wait(&bar_res[e], res_phase);  // every lane observes the phase itself
                     res_phase ^= 1u;

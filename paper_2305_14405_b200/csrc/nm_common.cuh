@@ -182,6 +182,30 @@ __device__ __forceinline__ bool nm_mbar_wait(uint64_t* bar, uint32_t parity, vol
     }
 }
 
+// The same bounded wait for warps that are NOT on the critical issue path (epilogue and
+// softmax warps waiting for the tensor core): between polls the thread sleeps, so that a
+// waiting warp does not take issue slots from the single thread that feeds the tensor core
+// on the same scheduler.
+__device__ __forceinline__ bool nm_mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                     int* status)
+{
+    if (nm_mbar_try_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    uint32_t spins = 0;
+    while (true) {
+        __nanosleep(40);
+        if (nm_mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > NM_WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, (int)NM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void nm_fence_barrier_init()
 {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
