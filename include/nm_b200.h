@@ -238,6 +238,31 @@ nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, i
                                 const nm_encoder_cfg* cfg, const void* x_host, void* y_host,
                                 void* x_dev, void* y_dev, void* workspace, size_t ws_bytes, void* stream);
 
+/* nm_encoder_layer for callers that cannot provide a workspace.  (The paper has no
+ * counterpart to this call: it exists for the library's users, not for the method.)
+ *
+ * Some callers have no way to allocate device memory: code that runs inside a host framework
+ * whose memory pool already owns the device's memory, a latency-critical serving loop in which
+ * cudaMalloc and its implicit device-wide synchronisation are off-limits, or a plug-in that
+ * receives only its input and output buffers.  For them the layer's scratch (the packed
+ * projection, attention output, pre-LayerNorm sums, FFN hidden activations) lives in a fixed
+ * array of NM_STATIC_WS_BYTES inside the library's device image; every GPU that loads the
+ * library holds that array until the process exits.  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating call; per-launch profiling records are suspended for its
+ * duration.  x, y, w, cfg, stream are exactly as in nm_encoder_layer.
+ *
+ * Limit: configurations with nm_encoder_workspace_bytes(cfg) > NM_STATIC_WS_BYTES return
+ * NM_ERR_WORKSPACE (use nm_encoder_layer with your own workspace for those).
+ * First call on a device resolves the array's device address (cudaGetSymbolAddress with that
+ * device made current for the moment); make that first call before starting any stream
+ * capture.  All calls on a device share the one array and it keeps the previous call's
+ * contents: nothing in it needs to start at zero (every buffer is fully written before it is
+ * read), but two calls whose kernels overlap on the GPU (different streams, no ordering
+ * between them) race on it. */
+#define NM_STATIC_WS_BYTES (32u << 20)
+nm_status nm_encoder_layer_static(nm_ctx* ctx, const nm_encoder_weights* w, const nm_encoder_cfg* cfg,
+                                  const void* x, void* y, void* stream);
+
 /* Number of kernels the library has launched through this context since creation
  * (or since the last call with reset != 0). */
 int64_t nm_ctx_launch_count(nm_ctx* ctx, int reset);

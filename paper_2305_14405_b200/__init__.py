@@ -20,12 +20,13 @@ F32, BF16, F16, I8 = 0, 1, 2, 3
 SLOT_NONE, SLOT_GELU, SLOT_EXP, SLOT_RECIP, SLOT_RSQRT, SLOT_RELU, SLOT_USER0 = -1, 0, 1, 2, 3, 4, 5
 FUNC_GELU, FUNC_EXP, FUNC_RECIP, FUNC_RSQRT, FUNC_RELU, FUNC_SQRT, FUNC_IDENTITY = range(7)
 ALGO_AUTO, ALGO_SIMT, ALGO_TC, ALGO_TC_1CTA = 0, 1, 2, 3
+STATIC_WS_BYTES = 32 << 20
 
 EXPORTS = [
     "nm_status_string", "nm_ctx_create", "nm_ctx_destroy", "nm_ctx_poll_status", "nm_ctx_launch_count",
     "nm_pwl_table_build", "nm_pwl_table_load", "nm_pwl_apply", "nm_linear_pwl", "nm_attention_pwl",
     "nm_layernorm_pwl", "nm_quantize_i8", "nm_encoder_workspace_bytes", "nm_encoder_layer", "nm_encoder_stack",
-    "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read",
+    "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
 ]
 KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc")
 
@@ -104,6 +105,8 @@ def load():
     lib.nm_encoder_stack_host.argtypes = [C.c_void_p, C.POINTER(EncoderWeights), C.c_int32, C.POINTER(EncoderCfg),
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                           C.c_void_p]
+    lib.nm_encoder_layer_static.argtypes = [C.c_void_p, C.POINTER(EncoderWeights), C.POINTER(EncoderCfg), C.c_void_p,
+                                            C.c_void_p, C.c_void_p]
     lib.nm_ctx_profile_enable.argtypes = [C.c_void_p, C.c_int]
     lib.nm_ctx_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_double),
                                         C.POINTER(C.c_double)]
@@ -297,6 +300,13 @@ class Context:
         _check(self._lib.nm_encoder_layer(self._h, C.byref(weights), C.byref(cfg), _ptr(x), _ptr(y),
                                           _ptr(workspace), workspace.numel() * workspace.element_size(),
                                           _stream(stream)), "nm_encoder_layer")
+
+    def encoder_layer_static(self, weights, cfg, x, y, stream=None):
+        """nm_encoder_layer_static: the layer with the library's own fixed scratch array instead of a
+        caller workspace, for callers that cannot allocate device memory.  Raises NmError
+        (NM_ERR_WORKSPACE) when the configuration needs more than STATIC_WS_BYTES."""
+        _check(self._lib.nm_encoder_layer_static(self._h, C.byref(weights), C.byref(cfg), _ptr(x), _ptr(y),
+                                                 _stream(stream)), "nm_encoder_layer_static")
 
     def encoder_stack(self, layer_array, n_layers, cfg, x, y, workspace, stream=None):
         _check(self._lib.nm_encoder_stack(self._h, layer_array, n_layers, C.byref(cfg), _ptr(x), _ptr(y),

@@ -448,3 +448,46 @@ nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, i
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------- encoder layer without a caller workspace
+//
+// Scratch for nm_encoder_layer_static: a fixed array in the library's own device image.  Every
+// GPU that loads the library carries these NM_STATIC_WS_BYTES until the process exits.
+// In host code the name `nm_static_ws` is only a handle for the runtime, not a device address:
+// the address a kernel may use is the one cudaGetSymbolAddress returns, per device.
+static __device__ __align__(256) unsigned char nm_static_ws[NM_STATIC_WS_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_ws_ptr[kMaxDevices];   // resolved device address of nm_static_ws, per device
+bool g_static_ws_ready[kMaxDevices];
+}  // namespace
+
+extern "C" nm_status nm_encoder_layer_static(nm_ctx* ctx, const nm_encoder_weights* w, const nm_encoder_cfg* cfg,
+                                             const void* x, void* y, void* stream)
+{
+    if (!ctx || !w || !cfg || !x || !y) return NM_ERR_INVALID_ARG;
+    const size_t need = nm_encoder_workspace_bytes(cfg);
+    if (need == 0) return NM_ERR_SHAPE;
+    if (need > (size_t)NM_STATIC_WS_BYTES) return NM_ERR_WORKSPACE;  // larger layers must bring their own workspace
+    const int dev = ctx->device;
+    if (dev < 0 || dev >= kMaxDevices) return NM_ERR_UNSUPPORTED;
+    if (!g_static_ws_ready[dev]) {
+        // first call on this device: resolve the array's device address with that device current
+        int cur = -1;
+        NM_CUDA_TRY(cudaGetDevice(&cur));
+        if (cur != dev) NM_CUDA_TRY(cudaSetDevice(dev));
+        void* p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&p, nm_static_ws);
+        if (cur != dev) cudaSetDevice(cur);
+        if (e != cudaSuccess || p == nullptr) return NM_ERR_CUDA;
+        g_static_ws_ptr[dev] = p;
+        g_static_ws_ready[dev] = true;
+    }
+    // per-launch event records (profiling) would create CUDA events: keep them off in this call
+    const int prof = ctx->profiling;
+    ctx->profiling = 0;
+    const nm_status s = nm_encoder_layer(ctx, w, cfg, x, y, g_static_ws_ptr[dev], (size_t)NM_STATIC_WS_BYTES, stream);
+    ctx->profiling = prof;
+    return s;
+}
