@@ -37,7 +37,7 @@ def parse_args():
     p.add_argument("--steps", type=int, default=100)
     p.add_argument("--warmup", type=int, default=10)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--workload", default="c3", choices=["c1", "c2", "c3"])
+    p.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4"])
     p.add_argument("--segments", type=int, default=64)
     p.add_argument("--seed", type=int, default=0)
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -152,7 +152,15 @@ def time_oracle(cfg, x, layers, n_layers, n_seq):
     L = cfg.L
     xin = x[: n_seq * L]
     t0 = time.perf_counter()
-    oracle.encoder_stack(xin, layers[:n_layers], n_seq, L, cfg.heads, tabs, cfg.eps)
+    if cfg.dtype == "i8":      # the int8 evaluation: same int8 weights and scales the GPU path receives
+        import nm_inputs
+        quant = nm_inputs.int8_encoder_inputs(cfg, layers[:n_layers])
+        t0 = time.perf_counter()
+        y = xin
+        for li in range(n_layers):
+            y = oracle.encoder_layer_i8(y, layers[li], quant[li], n_seq, L, cfg.heads, tabs, cfg.eps)
+    else:
+        oracle.encoder_stack(xin, layers[:n_layers], n_seq, L, cfg.heads, tabs, cfg.eps)
     dt = time.perf_counter() - t0
     full = dt * cfg.layers / n_layers
     return n_seq * L / full, dt, oracle.num_threads()
@@ -222,7 +230,8 @@ def main():
     x_np, layers_np = nm_inputs.encoder_inputs(cfg, seed=args.seed)
     if rank > 0:
         x_np, _ = nm_inputs.encoder_inputs(cfg, seed=args.seed + rank, layers=0)
-    model = EncoderModel(ctx, cfg, layers_np, device=dev, algo=args.algo)
+    quant = nm_inputs.int8_encoder_inputs(cfg, layers_np) if cfg.dtype == "i8" else None
+    model = EncoderModel(ctx, cfg, layers_np, device=dev, algo=args.algo, quant=quant)
     act = model.act_dtype()
     x = torch.from_numpy(x_np).to(dev).to(act)
     y = torch.empty_like(x)
@@ -297,7 +306,8 @@ def main():
         gemm_kind = "linear_tc" if prof["linear_tc"][0] else "linear_simt"
         n_l, ms_l, work_l = prof[gemm_kind]
         achieved = work_l / (ms_l * 1e-3) / 1e12 if ms_l > 0 else 0.0
-        peak = peaks["bf16_tflops_sustained"] if cfg.dtype != "f32" else peaks["bf16_tflops_sustained"] / 2
+        # int8: the measured bf16 peak times the nominal 2:1 int8:bf16 ratio; fp32 runs on CUDA cores
+        peak = {"i8": 2.0, "f32": 0.5}.get(cfg.dtype, 1.0) * peaks["bf16_tflops_sustained"]
         roofline = {"bound": "tensor", "kernel": gemm_kind, "achieved": achieved, "peak": peak,
                     "unit": "TFLOP/s", "frac": achieved / peak,
                     "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name),

@@ -144,3 +144,31 @@ def pwl_probe_points(x_min, x_max, n, count, seed):
     near = np.concatenate([bp, np.nextafter(bp, np.float32(np.inf)), np.nextafter(bp, np.float32(-np.inf))])
     special = np.array([0.0, -0.0, np.inf, -np.inf, 1e30, -1e30], np.float32)
     return np.concatenate([u, near, special]).astype(np.float32)
+
+
+def quantize_weights_per_channel(W: np.ndarray):
+    """Symmetric int8 per output channel (row): scale_j = max|W[j,:]| / 127, code = rint(W / scale) in
+    [-127, 127] (ties to even).  The int8 codes and fp32 scales ARE the inputs both sides receive."""
+    W = np.asarray(W, np.float32)
+    s = (np.abs(W).max(axis=1) / np.float32(127.0)).astype(np.float32)
+    s = np.maximum(s, np.float32(1e-12))
+    q = np.clip(np.rint(W / s[:, None]), -127, 127).astype(np.int8)
+    return q, s
+
+
+def int8_encoder_inputs(cfg: EncoderConfig, layers):
+    """Per-layer int8 weights, weight scales and static per-tensor activation scales for the int8 path.
+    Activation scales are fixed from the synthetic distributions (inputs and LayerNorm outputs ~N(0,1),
+    attention output ~N(0, 0.02^2 H / L), GELU output of N(0, 0.02^2 H)): the same numbers go to both sides."""
+    sig_v = 0.02 * np.sqrt(cfg.H)
+    scales = {"a_x": 5.5 / 127.0, "a_attn": 6.0 * sig_v / np.sqrt(cfg.L) / 127.0, "a_x1": 5.5 / 127.0,
+              "a_g": 4.5 * sig_v / 127.0}
+    out = []
+    for w in layers:
+        d = {k: float(np.float32(v)) for k, v in scales.items()}
+        for name in ("Wqkv", "Wo", "W1", "W2"):
+            q, s = quantize_weights_per_channel(w[name])
+            d[name + "_q"] = q
+            d[name + "_s"] = s
+        out.append(d)
+    return out

@@ -342,3 +342,38 @@ def avgpool_nhwc(x):
     out = np.empty((Nb, Cc))
     lib().nmo_avgpool_nhwc(_dp(x), C.c_int32(Nb), C.c_int32(Hin), C.c_int32(Win), C.c_int32(Cc), _dp(out))
     return out
+
+
+def encoder_layer_i8(x, w: dict, q: dict, B, L, h, tables: dict, eps=1e-5):
+    """The int8 evaluation of one encoder layer (Section 5 evaluates INT8 networks): the four weight
+    GEMMs take int8 activations (static per-tensor scales q['a_*']) and int8 weights (per-channel scales
+    q['W*_s']); everything between them is the fp64 path above.  Composition of the routines in this
+    file, in the order of nmo_encoder_layer:
+        qkv = deq(Q(x)) Wqkv^T + b;  a = attention(qkv);  x1 = LN(x + deq(Q(a)) Wo^T + bo)
+        g = PWLgelu(deq(Q(x1)) W1^T + b1);  y = LN(x1 + deq(Q(g)) W2^T + b2)
+    with Q(t) = clamp(rint(t / scale), -127, 127) and deq(c) = c * scale."""
+    x = _f64(x)
+
+    # A quantised code is an integer decided by a floating-point value; it is taken in the
+    # precision the workload stores that value in: activations between operators are bf16
+    # (round to nearest even), the GELU output is requantised from its fp32 epilogue value.
+    def bf16(t):
+        u = np.ascontiguousarray(t, dtype=np.float32).view(np.uint32)
+        r = ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000))
+        return r.view(np.float32).astype(np.float64)
+
+    def deq_act(t, scale):
+        return quantize_i8(np.asarray(t, np.float32), scale).astype(np.float64) * float(np.float32(scale))
+
+    def deq_w(name):
+        return q[name + "_q"].astype(np.float64) * q[name + "_s"].astype(np.float64)[:, None]
+
+    H = x.shape[1]
+    d = H // h
+    qkv = bf16(linear(deq_act(x, q["a_x"]), deq_w("Wqkv"), w["bqkv"]))
+    a = bf16(attention(qkv, B, L, h, d, tables["exp"], tables["recip"]))
+    z = bf16(linear(deq_act(a, q["a_attn"]), deq_w("Wo"), w["bo"], residual=x))
+    x1 = bf16(layernorm(z, w["g1"], w["be1"], eps, tables["rsqrt"]))
+    g = linear(deq_act(x1, q["a_x1"]), deq_w("W1"), w["b1"], table=tables["gelu"])
+    z2 = bf16(linear(deq_act(g, q["a_g"]), deq_w("W2"), w["b2"], residual=x1))
+    return layernorm(z2, w["g2"], w["be2"], eps, tables["rsqrt"])

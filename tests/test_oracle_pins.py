@@ -460,3 +460,39 @@ def test_alg3_bias_correction():
     k, b = oracle.secant_points(oracle.GELU, np.array([fx["alg3_biased_segment_from"], fx["alg3_biased_segment_to"]]))
     _, dE = oracle.bias_correct(oracle.GELU, np.array([-1.0, 0.0]), b)
     assert dE[0] < -0.02
+
+
+def test_int8_encoder_layer_against_library_routines():
+    """The int8 evaluation of a layer, rebuilt from library routines only (numpy rint/clip for the
+    quantiser, numpy matmul, torch attention / layer_norm / gelu in fp64, torch bf16 casts) with exact
+    nonlinearities: must agree with the oracle's composition in exact mode."""
+    cfg = nm_inputs.with_(nm_inputs.C4, B=2, L=24, H=64, heads=4, F=128, layers=1)
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=5, random_affine=True)
+    w = layers[0]
+    q = nm_inputs.int8_encoder_inputs(cfg, layers)[0]
+    got = oracle.encoder_layer_i8(x, w, q, cfg.B, cfg.L, cfg.heads, _exact_tables())
+
+    def bf(t):
+        return torch.from_numpy(np.asarray(t, np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+
+    def quant(t, s):
+        s32 = np.float32(s)
+        inv = np.float32(1.0) / s32
+        return np.clip(np.rint(np.asarray(t, np.float32) * inv), -127, 127).astype(np.float64) * float(s32)
+
+    def wdq(name):
+        return q[name + "_q"].astype(np.float64) * q[name + "_s"].astype(np.float64)[:, None]
+
+    H, h, d = cfg.H, cfg.heads, cfg.d
+    qkv = bf(quant(x, q["a_x"]) @ wdq("Wqkv").T + w["bqkv"])
+    a = bf(_torch_attention(qkv, cfg.B, cfg.L, h, d))
+    z = bf(quant(a, q["a_attn"]) @ wdq("Wo").T + w["bo"] + x)
+    ln = lambda t, g, b: torch.nn.functional.layer_norm(torch.from_numpy(t), (H,), torch.from_numpy(g.astype(np.float64)),
+                                                        torch.from_numpy(b.astype(np.float64)), 1e-5).numpy()
+    x1 = bf(ln(z, w["g1"], w["be1"]))
+    g = torch.nn.functional.gelu(torch.from_numpy(quant(x1, q["a_x1"]) @ wdq("W1").T + w["b1"])).numpy()
+    z2 = bf(quant(g, q["a_g"]) @ wdq("W2").T + w["b2"] + x1)
+    ref = ln(z2, w["g2"], w["be2"])
+    # a code on a rounding boundary may differ between two fp64 summation orders: allow a few elements
+    err = np.abs(got - ref)
+    assert (err > 1e-9).mean() < 0.02 and np.median(err) < 1e-12
