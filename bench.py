@@ -1,14 +1,17 @@
-"""Benchmark of the PWL BERT encoder forward pass on B200.
+"""Benchmark of the PWL forward pass on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c1] [--segments n]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c1|c4|c5] [--segments n]
     python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
 
-A step is one pass of the whole encoder stack (every layer: QKV GEMM, PWL attention,
-out-projection + residual, PWL LayerNorm, FFN1 + PWL GELU, FFN2 + residual, PWL LayerNorm)
-over one batch of seeded synthetic input.  Rank 0 prints one JSON line.
+Default workload c3: the 12-layer BERT-base-shaped PWL encoder (batch 32, seq 512), the
+configuration the metric "PWL BERT encoder tokens/s" is quoted on.  A step is one pass of the whole
+network over one batch of seeded synthetic input (encoder: per layer QKV GEMM, PWL attention,
+out-projection + residual, PWL LayerNorm, FFN1 + PWL GELU, FFN2 + residual, PWL LayerNorm; c5: the
+ResNet-50-shaped CNN, 53 convolutions as GEMMs with ReLU tables, pools, classifier).  Rank 0 prints
+one JSON line.
 
-The path has no exchange step: with N > 1 every rank runs an independent replica on its own
-batch (weak scaling, no collective on the data path); only the timing barrier is shared.
+The path has no exchange step: with N > 1 every rank runs an independent replica on its own batch
+(weak scaling, no collective on the data path); only the timing barrier is shared.
 """
 from __future__ import annotations
 
@@ -23,8 +26,6 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "PWL BERT encoder tokens/s"
-UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, mean over the four
 # GEMM shapes of a layer, from the ncu capture summarised in profiles/encoder_c3_launches_and_kernels.md
@@ -37,9 +38,10 @@ def parse_args():
     p.add_argument("--steps", type=int, default=100)
     p.add_argument("--warmup", type=int, default=10)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4"])
+    p.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
     p.add_argument("--segments", type=int, default=64)
     p.add_argument("--seed", type=int, default=0)
+    p.add_argument("--batch", type=int, default=0, help="override the batch size (c5 only)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--algo", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     return p.parse_args()
@@ -73,17 +75,9 @@ class ClockSampler(threading.Thread):
             nv.nvmlInit()
             h = nv.nvmlDeviceGetHandleByIndex(self.index)
             self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
-            names = {
-                getattr(nv, "nvmlClocksEventReasonGpuIdle", 0x1): "gpu_idle",
-                getattr(nv, "nvmlClocksEventReasonApplicationsClocksSetting", 0x2): "applications_clocks_setting",
-                getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
-                getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
-                getattr(nv, "nvmlClocksEventReasonSyncBoost", 0x10): "sync_boost",
-                getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
-                getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
-                getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
-                getattr(nv, "nvmlClocksEventReasonDisplayClockSetting", 0x100): "display_clock_setting",
-            }
+            names = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+                     0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+                     0x100: "display_clock_setting"}
             get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 nv.nvmlDeviceGetCurrentClocksThrottleReasons
             while not self._stop_evt.is_set():
@@ -94,7 +88,7 @@ class ClockSampler(threading.Thread):
                     pass
                 mask = get_reasons(h)
                 for bit, name in names.items():
-                    if mask & bit and name != "gpu_idle":
+                    if mask & bit:
                         self.reasons.add(name)
                 time.sleep(0.02)
         except Exception as e:  # NVML missing: report that rather than invent clocks
@@ -115,7 +109,7 @@ class ClockSampler(threading.Thread):
         return out
 
 
-def dist_setup(n):
+def dist_setup():
     import torch
     import torch.distributed as dist
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -137,104 +131,250 @@ def physical_gpu_index(local):
     return local
 
 
-def oracle_tables(cfg):
-    import oracle
-    r = cfg.ranges()
-    funcs = {"gelu": oracle.GELU, "exp": oracle.EXP, "recip": oracle.RECIP, "rsqrt": oracle.RSQRT}
-    return {k: oracle.Table.secant(funcs[k], cfg.segments, *r[k]) for k in funcs}
+# ----------------------------------------------------------------------------------------------
+# workloads
+# ----------------------------------------------------------------------------------------------
 
+class EncoderWorkload:
+    """c1..c4: the PWL transformer encoder stack; unit = tokens."""
+    metric = "PWL BERT encoder tokens/s"
+    unit = "tokens/s"
 
-def time_oracle(cfg, x, layers, n_layers, n_seq):
-    """Times the oracle, as it stands, on `n_seq` sequences through `n_layers` layers.
-    Returns (tokens/s of the FULL stack, seconds, threads)."""
-    import oracle
-    tabs = oracle_tables(cfg)
-    L = cfg.L
-    xin = x[: n_seq * L]
-    t0 = time.perf_counter()
-    if cfg.dtype == "i8":      # the int8 evaluation: same int8 weights and scales the GPU path receives
+    def __init__(self, args):
         import nm_inputs
-        quant = nm_inputs.int8_encoder_inputs(cfg, layers[:n_layers])
+        self.args = args
+        self.cfg = nm_inputs.with_(nm_inputs.CONFIGS[args.workload], segments=args.segments)
+        self.dtype = self.cfg.dtype
+        self.units_per_step = self.cfg.T
+
+    def config(self, world):
+        c = self.cfg
+        return {"workload": c.name, "layers": c.layers, "batch": c.B, "seq_len": c.L, "hidden": c.H, "heads": c.heads,
+                "ffn": c.F, "pwl_segments": c.segments, "seed": self.args.seed,
+                "parallelism": "replicas" if world > 1 else "single",
+                "l2": "working set per step (weights %.0f MB + activations %.0f MB) exceeds the 126 MB L2; no flush"
+                      % (c.layers * (4 * c.H * c.H + 2 * c.H * c.F) * (1 if c.dtype == "i8" else 2) / 1e6,
+                         c.T * (6 * c.H + c.F) * 2 / 1e6)}
+
+    def flops_per_step(self):
+        return self.cfg.layers * self.cfg.flops_per_layer()
+
+    def setup(self, ctx, dev, rank):
+        import torch
+        import nm_inputs
+        from paper_2305_14405_b200.harness import EncoderModel
+        cfg = self.cfg
+        ctx.load_encoder_tables(cfg.segments, cfg.ranges())
+        self.x_np, self.layers_np = nm_inputs.encoder_inputs(cfg, seed=self.args.seed)
+        if rank > 0:  # every rank draws its own batch: independent replicas of the same model
+            self.x_np, _ = nm_inputs.encoder_inputs(cfg, seed=self.args.seed + rank, layers=0)
+        quant = nm_inputs.int8_encoder_inputs(cfg, self.layers_np) if cfg.dtype == "i8" else None
+        self.model = EncoderModel(ctx, cfg, self.layers_np, device=dev, algo=self.args.algo, quant=quant)
+        act = self.model.act_dtype()
+        self.x = torch.from_numpy(self.x_np).to(dev).to(act)
+        self.y = torch.empty_like(self.x)
+        self.xh = torch.from_numpy(self.x_np).to(act).pin_memory()
+        self.yh = torch.empty_like(self.xh).pin_memory()
+        self.ctx = ctx
+        self.h2d = self.d2h = cfg.T * cfg.H * self.x.element_size()
+
+    def step(self):
+        self.model.forward(self.x, self.y)
+
+    def host_step(self):
+        m = self.model
+        self.ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, self.xh, self.yh, self.x, self.y, m.workspace)
+
+    # -- the oracle, as it stands, on whole sampled sequences (sequences are independent) -----------
+    def _oracle_tables(self):
+        import oracle
+        r = self.cfg.ranges()
+        funcs = {"gelu": oracle.GELU, "exp": oracle.EXP, "recip": oracle.RECIP, "rsqrt": oracle.RSQRT}
+        return {k: oracle.Table.secant(funcs[k], self.cfg.segments, *r[k]) for k in funcs}
+
+    def time_oracle(self, x, layers, n_layers, n_seq):
+        """Returns (units/s of the FULL stack, seconds, threads)."""
+        import oracle
+        cfg = self.cfg
+        tabs = self._oracle_tables()
+        xin = x[: n_seq * cfg.L]
+        if cfg.dtype == "i8":  # the int8 evaluation: same int8 weights and scales the GPU path receives
+            import nm_inputs
+            quant = nm_inputs.int8_encoder_inputs(cfg, layers[:n_layers])
+            t0 = time.perf_counter()
+            y = xin
+            for li in range(n_layers):
+                y = oracle.encoder_layer_i8(y, layers[li], quant[li], n_seq, cfg.L, cfg.heads, tabs, cfg.eps)
+        else:
+            t0 = time.perf_counter()
+            oracle.encoder_stack(xin, layers[:n_layers], n_seq, cfg.L, cfg.heads, tabs, cfg.eps)
+        dt = time.perf_counter() - t0
+        return n_seq * cfg.L / (dt * cfg.layers / n_layers), dt, oracle.num_threads()
+
+    def cpu_baseline(self):
+        cfg = self.cfg
+        _, t1, _ = self.time_oracle(self.x_np, self.layers_np, 1, 1)   # calibrate, then ~15 s of CPU work
+        n_layers = max(1, min(cfg.layers, int(15.0 / max(t1, 1e-3))))
+        n_seq = max(1, min(cfg.B, int(15.0 / max(t1 * n_layers, 1e-3))))
+        v, secs, cores = self.time_oracle(self.x_np, self.layers_np, n_layers, n_seq)
+        return {"value": v, "unit": self.unit, "cores": cores, "kind": "oracle",
+                "sample": "%d of %d sequences (%d tokens each) through %d of %d layers, %.1f s%s"
+                          % (n_seq, cfg.B, cfg.L, n_layers, cfg.layers, secs,
+                             "" if n_layers == cfg.layers else "; scaled by the layer count")}
+
+    def reference_setup(self):
+        import nm_inputs
+        self.x_np, self.layers_np = nm_inputs.encoder_inputs(self.cfg, seed=self.args.seed, layers=1)
+        self.ref_sample = "1 of %d sequences (%d tokens) through 1 of %d layers per step, scaled by the layer count" % (
+            self.cfg.B, self.cfg.L, self.cfg.layers)
+
+    def reference_step(self):
+        """Runs one bounded sample; returns the units of full-network work it stands for."""
+        self.time_oracle(self.x_np, self.layers_np, 1, 1)
+        return self.cfg.L / self.cfg.layers
+
+
+class ResnetWorkload:
+    """c5: the ResNet-50-shaped CNN run as GEMMs with ReLU tables, fp16 NHWC; unit = images."""
+    metric = "PWL ResNet-50 images/s"
+    unit = "images/s"
+    dtype = "f16"
+
+    def __init__(self, args):
+        self.args = args
+        self.batch = args.batch or 128
+        self.units_per_step = self.batch
+
+    def config(self, world):
+        return {"workload": "c5_resnet50_f16", "batch": self.batch, "image": "224x224x3 NHWC", "convolutions": 53,
+                "classes": 1000, "batchnorm": "folded into weights and biases", "relu": "2-segment PWL table",
+                "seed": self.args.seed, "parallelism": "replicas" if world > 1 else "single",
+                "l2": "activations (up to %.0f MB per layer at this batch) exceed the 126 MB L2; no flush"
+                      % (self.batch * 112 * 112 * 64 * 2 / 1e6)}
+
+    def flops_per_step(self):
+        import nm_inputs_cnn
+        specs = iter(nm_inputs_cnn.resnet50_conv_specs())
+        cin, cout, k, _, _ = next(specs)
+        total = 2 * 112 * 112 * cout * k * k * cin
+        h = 56
+        for st, nb in enumerate(nm_inputs_cnn.STAGE_BLOCKS):
+            for b in range(nb):
+                stride = 2 if (b == 0 and st > 0) else 1
+                ho = h // stride
+                ca, cb, cc = next(specs), next(specs), next(specs)
+                total += 2 * h * h * ca[1] * ca[0] + 2 * ho * ho * cb[1] * 9 * cb[0] + 2 * ho * ho * cc[1] * cc[0]
+                if b == 0:
+                    cd = next(specs)
+                    total += 2 * ho * ho * cd[1] * cd[0]
+                h = ho
+        total += 2 * 2048 * 1000
+        return total * self.batch
+
+    def setup(self, ctx, dev, rank):
+        import torch
+        import nm_inputs_cnn
+        import paper_2305_14405_b200 as nm
+        from paper_2305_14405_b200.harness_cnn import Resnet50Model
+        ctx.load_function_table(nm.SLOT_RELU, nm.FUNC_RELU, 2, -8.0, 8.0)
+        # the same model on every replica (seed), its own images per rank (seed + rank)
+        self.x_np, self.convs, self.fc_w, self.fc_b = nm_inputs_cnn.resnet50_inputs(
+            self.batch, seed=self.args.seed, random_bn=True)
+        if rank > 0:
+            import numpy as np
+            import nm_inputs
+            rng = np.random.default_rng(self.args.seed + rank)
+            self.x_np = nm_inputs.round_to(rng.random(self.x_np.shape, dtype=np.float32), "f16")
+        self.model = Resnet50Model(ctx, self.batch, self.convs, self.fc_w, self.fc_b, device=dev, algo=self.args.algo)
+        self.x = torch.from_numpy(self.x_np).to(dev).half()
+        self.y = torch.empty((self.batch, 1000), dtype=torch.float16, device=dev)
+        self.xh = torch.from_numpy(self.x_np).half().pin_memory()
+        self.yh = torch.empty((self.batch, 1000), dtype=torch.float16).pin_memory()
+        self.ctx = ctx
+        self.h2d = self.batch * 224 * 224 * 3 * 2
+        self.d2h = self.batch * 1000 * 2
+
+    def step(self):
+        self.model.forward(self.x, self.y)
+
+    def host_step(self):
+        m = self.model
+        self.ctx.resnet50_forward_host(m.array, m.fc_w, m.fc_b, m.cfg, self.xh, self.yh, self.x, self.y, m.workspace)
+
+    def _oracle_run(self, n_img):
+        import oracle
+        import oracle.cnn
+        relu = oracle.Table.secant(oracle.RELU, 2, -8.0, 8.0)
         t0 = time.perf_counter()
-        y = xin
-        for li in range(n_layers):
-            y = oracle.encoder_layer_i8(y, layers[li], quant[li], n_seq, L, cfg.heads, tabs, cfg.eps)
-    else:
-        oracle.encoder_stack(xin, layers[:n_layers], n_seq, L, cfg.heads, tabs, cfg.eps)
-    dt = time.perf_counter() - t0
-    full = dt * cfg.layers / n_layers
-    return n_seq * L / full, dt, oracle.num_threads()
+        oracle.cnn.resnet50(self.x_np[:n_img], self.convs, self.fc_w, self.fc_b, relu)
+        return time.perf_counter() - t0, oracle.num_threads()
+
+    def cpu_baseline(self):
+        t1, cores = self._oracle_run(1)
+        n = max(1, min(self.batch, int(15.0 / max(t1, 1e-3))))
+        secs, cores = self._oracle_run(n)
+        return {"value": n / secs, "unit": self.unit, "cores": cores, "kind": "oracle",
+                "sample": "%d of %d images through the whole network, %.1f s" % (n, self.batch, secs)}
+
+    def reference_setup(self):
+        import nm_inputs_cnn
+        self.x_np, self.convs, self.fc_w, self.fc_b = nm_inputs_cnn.resnet50_inputs(1, seed=self.args.seed, random_bn=True)
+        self.ref_sample = "1 of %d images through the whole network per step" % self.batch
+
+    def reference_step(self):
+        self._oracle_run(1)
+        return 1.0
 
 
-def run_reference(args, cfg):
-    """The CPU oracle on the host cores; one step = one sequence through one layer (a bounded
-    sample), scaled by the layer count to the metric's unit."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+def make_workload(args):
+    return ResnetWorkload(args) if args.workload == "c5" else EncoderWorkload(args)
+
+
+def run_reference(args, wl):
+    """The CPU oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    import nm_inputs
     import oracle
-    x, layers = nm_inputs.encoder_inputs(cfg, seed=args.seed, layers=1)
+    wl.reference_setup()
     for _ in range(args.warmup):
-        time_oracle(cfg, x, layers, 1, 1)
+        wl.reference_step()
     t0 = time.perf_counter()
+    units = 0.0
     for _ in range(args.steps):
-        time_oracle(cfg, x, layers, 1, 1)
-    dt = (time.perf_counter() - t0) / max(args.steps, 1)
-    value = cfg.L / (dt * cfg.layers)
-    sample = "1 of %d sequences (%d tokens) through 1 of %d layers per step, scaled by the layer count" % (
-        cfg.B, cfg.L, cfg.layers)
+        units += wl.reference_step()
+    dt = time.perf_counter() - t0
+    value = units / dt
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(cfg, args),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                         "sample": sample},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "impl": "reference", "metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": wl.config(1),
+        "cpu_baseline": {"value": value, "unit": wl.unit, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": wl.ref_sample},
+        "e2e": {"value": value, "unit": wl.unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
-def workload_config(cfg, args):
-    return {"workload": cfg.name, "layers": cfg.layers, "batch": cfg.B, "seq_len": cfg.L, "hidden": cfg.H,
-            "heads": cfg.heads, "ffn": cfg.F, "pwl_segments": cfg.segments, "seed": args.seed,
-            "parallelism": "replicas" if args.gpus > 1 else "single",
-            "l2": "working set per step (weights %.0f MB + activations %.0f MB) exceeds the 126 MB L2; no flush"
-                  % (cfg.layers * (4 * cfg.H * cfg.H + 2 * cfg.H * cfg.F) * 2 / 1e6,
-                     cfg.T * (6 * cfg.H + cfg.F) * 2 / 1e6)}
-
-
 def main():
     args = parse_args()
-    import nm_inputs
-    cfg = nm_inputs.with_(nm_inputs.CONFIGS[args.workload], segments=args.segments)
+    wl = make_workload(args)
     if args.impl == "reference":
-        run_reference(args, cfg)
+        run_reference(args, wl)
         return
 
     import torch
     import torch.distributed as dist
     import paper_2305_14405_b200 as nm
-    from paper_2305_14405_b200.harness import EncoderModel
 
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
-    world, rank, local = dist_setup(args.gpus)
+    world, rank, local = dist_setup()
     dev = "cuda:%d" % local
     torch.cuda.set_device(local)
     nm.load()
     ctx = nm.Context(local)
-    ctx.load_encoder_tables(cfg.segments, cfg.ranges())
-    # every rank draws its own batch (seed + rank): independent replicas of the same model
-    x_np, layers_np = nm_inputs.encoder_inputs(cfg, seed=args.seed)
-    if rank > 0:
-        x_np, _ = nm_inputs.encoder_inputs(cfg, seed=args.seed + rank, layers=0)
-    quant = nm_inputs.int8_encoder_inputs(cfg, layers_np) if cfg.dtype == "i8" else None
-    model = EncoderModel(ctx, cfg, layers_np, device=dev, algo=args.algo, quant=quant)
-    act = model.act_dtype()
-    x = torch.from_numpy(x_np).to(dev).to(act)
-    y = torch.empty_like(x)
+    wl.setup(ctx, dev, rank)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -242,8 +382,15 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        model.forward(x, y)
+    def max_over_ranks(ms):
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        wl.step()
     ctx.check_device_status()
 
     # ---- timed region: K steps, CUDA events on the launching stream ------------------------
@@ -256,47 +403,37 @@ def main():
     barrier()
     ev0.record(stream)
     for _ in range(args.steps):
-        model.forward(x, y)
+        wl.step()
     ev1.record(stream)
     barrier()
-    ms_total = ev0.elapsed_time(ev1)
+    ms_step = max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
     launches = ctx.launch_count()
     sampler.stop()
     ctx.check_device_status()
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    ms_step = ms_total / args.steps
-    value = world * cfg.T / (ms_step * 1e-3)
+    value = world * wl.units_per_step / (ms_step * 1e-3)
 
     # ---- per-kernel pass: the same steps with every launch bracketed by events -------------
-    prof_steps = min(args.steps, max(1, 8000 // max(1, launches // max(args.steps, 1))))
+    per_step = max(1, launches // max(args.steps, 1))
+    prof_steps = min(args.steps, max(1, 8000 // per_step))
     ctx.profile_enable(True)
     for _ in range(prof_steps):
-        model.forward(x, y)
+        wl.step()
     torch.cuda.synchronize()
     prof = ctx.profile_read()
     ctx.profile_enable(False)
 
     # ---- end to end through the C ABI with host buffers ------------------------------------
-    xh = torch.from_numpy(x_np).to(act).pin_memory()
-    yh = torch.empty_like(xh).pin_memory()
     e2e_steps = max(3, min(args.steps, 20))
-    ctx.encoder_stack_host(model.array, model.n_layers, model.ccfg, xh, yh, x, y, model.workspace)
+    wl.host_step()
     barrier()
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(e2e_steps):
-        ctx.encoder_stack_host(model.array, model.n_layers, model.ccfg, xh, yh, x, y, model.workspace)
+        wl.host_step()
     e1.record(stream)
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / e2e_steps
-    act_bytes = cfg.T * cfg.H * x.element_size()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
 
     if rank == 0:
         peaks, peak_kind = load_peaks()
@@ -307,49 +444,40 @@ def main():
         n_l, ms_l, work_l = prof[gemm_kind]
         achieved = work_l / (ms_l * 1e-3) / 1e12 if ms_l > 0 else 0.0
         # int8: the measured bf16 peak times the nominal 2:1 int8:bf16 ratio; fp32 runs on CUDA cores
-        peak = {"i8": 2.0, "f32": 0.5}.get(cfg.dtype, 1.0) * peaks["bf16_tflops_sustained"]
+        peak = {"i8": 2.0, "f32": 0.5}.get(wl.dtype, 1.0) * peaks["bf16_tflops_sustained"]
+        cfg_name = wl.config(world)["workload"]
         roofline = {"bound": "tensor", "kernel": gemm_kind, "achieved": achieved, "peak": peak,
                     "unit": "TFLOP/s", "frac": achieved / peak,
-                    "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name),
+                    "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg_name),
                     "peak_source": "%s (bf16 sustained: kernel timed inside a long step)" % peak_kind,
                     "avg_launch_us": ms_l / max(n_l, 1) * 1e3, "share_of_step": ms_l / total_ms}
         extra = {}
-        n_ln, ms_ln, work_ln = prof["layernorm"]
-        if n_ln:
-            gbs = work_ln / (ms_ln * 1e-3) / 1e9
-            extra["layernorm"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                  "frac": gbs / peaks["hbm_gbs"], "note": "algorithmic bytes; input is L2-resident "
-                                  "after the producing GEMM at this size"}
+        for kind in ("layernorm", "quantize", "im2col", "pool"):
+            n_k, ms_k, work_k = prof[kind]
+            if n_k:
+                gbs = work_k / (ms_k * 1e-3) / 1e9
+                extra[kind] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": gbs / peaks["hbm_gbs"], "note": "algorithmic bytes per launch / event time"}
         for kind in ("attention_tc", "attention_simt"):
             n_a, ms_a, work_a = prof[kind]
             if n_a:
                 tf = work_a / (ms_a * 1e-3) / 1e12
                 extra[kind] = {"bound": "alu", "achieved_tensor_tflops": tf, "avg_launch_us": ms_a / n_a * 1e3}
-        whole = cfg.layers * cfg.flops_per_layer() / (ms_step * 1e-3) / 1e12
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": workload_config(cfg, args),
+            "metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config(world),
             "clocks": sampler.summary(),
-            "e2e": {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": act_bytes,
-                    "d2h_bytes_per_step": act_bytes, "ms_per_step": e2e_ms},
+            "e2e": {"value": world * wl.units_per_step / (e2e_ms * 1e-3), "unit": wl.unit,
+                    "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": e2e_ms},
             "gpu_launches": launches,
             "roofline": roofline,
             "roofline_other": extra,
             "kernels": kernels,
-            "whole_step_tflops": whole,
+            "whole_step_tflops": wl.flops_per_step() / (ms_step * 1e-3) / 1e12,
         }
         if not args.no_cpu_baseline and world == 1:
-            # calibrate on one sequence through one layer, then size the sample to ~15 s of CPU work
-            _, t1, _ = time_oracle(cfg, x_np, layers_np, 1, 1)
-            n_layers = max(1, min(cfg.layers, int(15.0 / max(t1, 1e-3))))
-            n_seq = max(1, min(cfg.B, int(15.0 / max(t1 * n_layers, 1e-3))))
-            v, secs, cores = time_oracle(cfg, x_np, layers_np, n_layers, n_seq)
-            line["cpu_baseline"] = {
-                "value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                "sample": "%d of %d sequences (%d tokens each) through %d of %d layers, %.1f s%s"
-                          % (n_seq, cfg.B, cfg.L, n_layers, cfg.layers, secs,
-                             "" if n_layers == cfg.layers else "; scaled by the layer count")}
+            line["cpu_baseline"] = wl.cpu_baseline()
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

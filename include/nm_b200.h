@@ -140,6 +140,7 @@ typedef struct {
     int32_t* acc_dump;
     int32_t* idx_dump;
     int32_t algo;
+    int32_t res_first;  /* nonzero: out = PWL(A.W^T*scale + bias + residual), the order a ResNet block needs */
 } nm_linear_desc;
 
 nm_status nm_linear_pwl(nm_ctx* ctx, const nm_linear_desc* desc, void* stream);
@@ -238,6 +239,74 @@ nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, i
                                 const nm_encoder_cfg* cfg, const void* x_host, void* y_host,
                                 void* x_dev, void* y_dev, void* workspace, size_t ws_bytes, void* stream);
 
+/* 2-D convolution with PWL epilogue, NHWC (Section 3.1: convolution kernels are linear
+ * operations whose matrix dimensions follow from width, height and channels; Section 3: ReLU
+ * is already piecewise linear and is evaluated as a 2-segment table):
+ *     out[n,oy,ox,co] = PWL( sum_{ky,kx,ci} x[n, oy*stride-pad+ky, ox*stride-pad+kx, ci] * w[co,ky,kx,ci]
+ *                            + bias[co] ) + residual[n,oy,ox,co]          (zero padding)
+ * or, with res_first != 0, PWL( ... + bias + residual ), the order of a ResNet block.
+ * x [N,H,W,Cin], w [Cout,kh,kw,Cin], residual / out [N,Ho,Wo,Cout] with Ho = (H+2*pad-kh)/stride+1:
+ * device pointers of dtype (F16 or BF16), 16-byte aligned; bias device float[Cout] or NULL
+ * (BatchNorm is expected to be folded into w and bias by the caller).  Cout a multiple of 8;
+ * Cin a multiple of 8, except that any Cin is taken by the gather path (kh*kw*Cin is then
+ * padded to a multiple of 8).  It runs as a GEMM with M = N*Ho*Wo, K = kh*kw*Cin: 1x1 stride-1
+ * convolutions read x directly, all others first gather their operand into `workspace`
+ * (device, 256-byte aligned, at least nm_conv2d_workspace_bytes). */
+typedef struct {
+    int32_t N, H, W, Cin, Cout, kh, kw, stride, pad;
+    nm_dtype dtype;
+    const void* x;
+    const void* w;
+    const float* bias;
+    const void* residual;
+    int32_t slot;
+    int32_t res_first;
+    void* out;
+    int32_t algo;
+} nm_conv_desc;
+
+size_t nm_conv2d_workspace_bytes(const nm_conv_desc* desc);
+nm_status nm_conv2d_pwl(nm_ctx* ctx, const nm_conv_desc* desc, void* workspace, size_t ws_bytes, void* stream);
+
+/* Max pooling, NHWC, window ks x ks, zero-size padding cells ignored (a maximum is itself
+ * piecewise linear: max(a,b) = b + ReLU(a-b), Section 3), and global average pooling
+ * [N,H,W,C] -> [N,C] (a linear operator, Section 3.1: multiplication by a constant 1/(H*W)
+ * matrix; executed on CUDA cores because its operand is channel-contiguous).  C a multiple of 8. */
+nm_status nm_maxpool2d(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,
+                       int32_t C, int32_t ks, int32_t stride, int32_t pad, void* stream);
+nm_status nm_avgpool_global(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,
+                            int32_t C, void* stream);
+
+/* ResNet-50-shaped CNN computed entirely with GEMMs and PWL tables (Section 5 evaluates ResNet):
+ * 7x7/2 convolution, 3x3/2 max-pool, 16 bottleneck blocks (1x1 -> 3x3 -> 1x1, widths 64/128/256/512
+ * x4, the stride in the 3x3 convolution, 1x1 projection shortcut in the first block of a stage,
+ * ReLU after every convolution and after the residual add), global average pool, fully connected.
+ * convs: HOST array of NM_RESNET50_CONVS entries (device pointers inside) in network order:
+ * conv1, then per block conv_a, conv_b, conv_c and, for the first block of a stage, the shortcut
+ * projection.  x [batch,224,224,3] -> logits [batch, num_classes] of dtype (F16 or BF16);
+ * num_classes a multiple of 8. */
+#define NM_RESNET50_CONVS 53
+typedef struct {
+    const void* w;      /* [Cout, kh, kw, Cin] */
+    const float* bias;  /* [Cout] */
+} nm_conv_params;
+typedef struct {
+    int32_t batch;
+    nm_dtype dtype;
+    int32_t relu_slot;
+    int32_t num_classes;
+    int32_t algo;
+} nm_resnet50_cfg;
+size_t nm_resnet50_workspace_bytes(const nm_resnet50_cfg* cfg);
+nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w, const float* fc_b,
+                              const nm_resnet50_cfg* cfg, const void* x, void* logits, void* workspace,
+                              size_t ws_bytes, void* stream);
+/* The same with HOST input and output: x_host [batch,224,224,3] is copied to x_dev, the network
+ * runs, logits_dev is copied to logits_host, and the call waits for the stream. */
+nm_status nm_resnet50_forward_host(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w, const float* fc_b,
+                                   const nm_resnet50_cfg* cfg, const void* x_host, void* logits_host, void* x_dev,
+                                   void* logits_dev, void* workspace, size_t ws_bytes, void* stream);
+
 /* nm_encoder_layer for callers that cannot provide a workspace.  (The paper has no
  * counterpart to this call: it exists for the library's users, not for the method.)
  *
@@ -277,7 +346,8 @@ int64_t nm_ctx_launch_count(nm_ctx* ctx, int reset);
  * operator, 4*B*heads*L*L*d for attention) for the tensor-core-bound kinds, bytes
  * read plus written (one pass each way) for the bandwidth-bound row kernels. */
 enum { NM_KERNEL_PWL_APPLY = 0, NM_KERNEL_LAYERNORM = 1, NM_KERNEL_QUANTIZE = 2, NM_KERNEL_LINEAR_SIMT = 3,
-       NM_KERNEL_LINEAR_TC = 4, NM_KERNEL_ATTENTION_SIMT = 5, NM_KERNEL_ATTENTION_TC = 6, NM_NUM_KERNEL_KINDS = 7 };
+       NM_KERNEL_LINEAR_TC = 4, NM_KERNEL_ATTENTION_SIMT = 5, NM_KERNEL_ATTENTION_TC = 6, NM_KERNEL_IM2COL = 7,
+       NM_KERNEL_POOL = 8, NM_NUM_KERNEL_KINDS = 9 };
 nm_status nm_ctx_profile_enable(nm_ctx* ctx, int on);
 nm_status nm_ctx_profile_read(nm_ctx* ctx, int kind, int64_t* launches, double* total_ms, double* total_work);
 

@@ -27,8 +27,12 @@ EXPORTS = [
     "nm_pwl_table_build", "nm_pwl_table_load", "nm_pwl_apply", "nm_linear_pwl", "nm_attention_pwl",
     "nm_layernorm_pwl", "nm_quantize_i8", "nm_encoder_workspace_bytes", "nm_encoder_layer", "nm_encoder_stack",
     "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
+    "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
+    "nm_resnet50_forward", "nm_resnet50_forward_host",
 ]
-KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc")
+KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc",
+                "im2col", "pool")
+RESNET50_CONVS = 53
 
 
 class NmError(RuntimeError):
@@ -42,7 +46,8 @@ class LinearDesc(C.Structure):
                 ("A", C.c_void_p), ("lda", C.c_int64), ("W", C.c_void_p), ("ldw", C.c_int64), ("bias", C.c_void_p),
                 ("residual", C.c_void_p), ("ldr", C.c_int64), ("slot", C.c_int32), ("out", C.c_void_p),
                 ("ldo", C.c_int64), ("a_scale", C.c_float), ("w_scale", C.c_void_p), ("inv_out_scale", C.c_float),
-                ("acc_dump", C.c_void_p), ("idx_dump", C.c_void_p), ("algo", C.c_int32)]
+                ("acc_dump", C.c_void_p), ("idx_dump", C.c_void_p), ("algo", C.c_int32),
+                ("res_first", C.c_int32)]
 
 
 class AttnDesc(C.Structure):
@@ -58,6 +63,22 @@ class EncoderWeights(C.Structure):
                 ("W2", C.c_void_p), ("b2", C.c_void_p), ("g2", C.c_void_p), ("be2", C.c_void_p),
                 ("s_wqkv", C.c_void_p), ("s_wo", C.c_void_p), ("s_w1", C.c_void_p), ("s_w2", C.c_void_p),
                 ("a_x", C.c_float), ("a_attn", C.c_float), ("a_x1", C.c_float), ("a_g", C.c_float)]
+
+
+class ConvDesc(C.Structure):
+    _fields_ = [("N", C.c_int32), ("H", C.c_int32), ("W", C.c_int32), ("Cin", C.c_int32), ("Cout", C.c_int32),
+                ("kh", C.c_int32), ("kw", C.c_int32), ("stride", C.c_int32), ("pad", C.c_int32), ("dtype", C.c_int),
+                ("x", C.c_void_p), ("w", C.c_void_p), ("bias", C.c_void_p), ("residual", C.c_void_p),
+                ("slot", C.c_int32), ("res_first", C.c_int32), ("out", C.c_void_p), ("algo", C.c_int32)]
+
+
+class ConvParams(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("bias", C.c_void_p)]
+
+
+class Resnet50Cfg(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("dtype", C.c_int), ("relu_slot", C.c_int32), ("num_classes", C.c_int32),
+                ("algo", C.c_int32)]
 
 
 class EncoderCfg(C.Structure):
@@ -107,6 +128,19 @@ def load():
                                           C.c_void_p]
     lib.nm_encoder_layer_static.argtypes = [C.c_void_p, C.POINTER(EncoderWeights), C.POINTER(EncoderCfg), C.c_void_p,
                                             C.c_void_p, C.c_void_p]
+    lib.nm_conv2d_workspace_bytes.restype = C.c_size_t
+    lib.nm_conv2d_workspace_bytes.argtypes = [C.POINTER(ConvDesc)]
+    lib.nm_conv2d_pwl.argtypes = [C.c_void_p, C.POINTER(ConvDesc), C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.nm_maxpool2d.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_int32] * 7 + [C.c_void_p]
+    lib.nm_avgpool_global.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_int32] * 4 + [C.c_void_p]
+    lib.nm_resnet50_workspace_bytes.restype = C.c_size_t
+    lib.nm_resnet50_workspace_bytes.argtypes = [C.POINTER(Resnet50Cfg)]
+    lib.nm_resnet50_forward.argtypes = [C.c_void_p, C.POINTER(ConvParams), C.c_void_p, C.c_void_p,
+                                        C.POINTER(Resnet50Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                        C.c_void_p]
+    lib.nm_resnet50_forward_host.argtypes = [C.c_void_p, C.POINTER(ConvParams), C.c_void_p, C.c_void_p,
+                                             C.POINTER(Resnet50Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_size_t, C.c_void_p]
     lib.nm_ctx_profile_enable.argtypes = [C.c_void_p, C.c_int]
     lib.nm_ctx_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_double),
                                         C.POINTER(C.c_double)]
@@ -223,7 +257,7 @@ class Context:
                                       _stream(stream)), "nm_pwl_apply")
 
     def linear_pwl(self, A, W, out, bias=None, residual=None, slot=SLOT_NONE, a_scale=0.0, w_scale=None,
-                   inv_out_scale=0.0, acc_dump=None, idx_dump=None, algo=ALGO_AUTO, stream=None):
+                   inv_out_scale=0.0, acc_dump=None, idx_dump=None, algo=ALGO_AUTO, res_first=False, stream=None):
         d = LinearDesc()
         d.M, d.K = A.shape
         d.N = W.shape[0]
@@ -242,6 +276,7 @@ class Context:
         d.acc_dump = acc_dump.data_ptr() if acc_dump is not None else None
         d.idx_dump = idx_dump.data_ptr() if idx_dump is not None else None
         d.algo = algo
+        d.res_first = 1 if res_first else 0
         _check(self._lib.nm_linear_pwl(self._h, C.byref(d), _stream(stream)), "nm_linear_pwl")
 
     def attention_pwl(self, qkv, out, B, L, heads, d, scale=None, exp_slot=SLOT_EXP, recip_slot=SLOT_RECIP,
@@ -269,6 +304,64 @@ class Context:
     def quantize_i8(self, x, inv_scale, q, stream=None):
         _check(self._lib.nm_quantize_i8(self._h, _ptr(x), dtype_of(x), x.numel(), inv_scale, _ptr(q),
                                         _stream(stream)), "nm_quantize_i8")
+
+    # -- CNN ----------------------------------------------------------------------
+    @staticmethod
+    def conv_desc(x, w, out, stride, pad, bias=None, residual=None, slot=SLOT_NONE, res_first=False,
+                  algo=ALGO_AUTO):
+        """x [N,H,W,Cin], w [Cout,kh,kw,Cin], out [N,Ho,Wo,Cout] (contiguous device tensors)."""
+        d = ConvDesc()
+        d.N, d.H, d.W, d.Cin = x.shape
+        d.Cout, d.kh, d.kw = w.shape[0], w.shape[1], w.shape[2]
+        d.stride, d.pad = stride, pad
+        d.dtype = dtype_of(x)
+        d.x, d.w, d.out = x.data_ptr(), w.data_ptr(), out.data_ptr()
+        d.bias = bias.data_ptr() if bias is not None else None
+        d.residual = residual.data_ptr() if residual is not None else None
+        d.slot = slot
+        d.res_first = 1 if res_first else 0
+        d.algo = algo
+        return d
+
+    def conv2d_workspace_bytes(self, desc) -> int:
+        return int(self._lib.nm_conv2d_workspace_bytes(C.byref(desc)))
+
+    def conv2d_pwl(self, desc, workspace=None, stream=None):
+        ws = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        _check(self._lib.nm_conv2d_pwl(self._h, C.byref(desc), _ptr(workspace), ws, _stream(stream)), "nm_conv2d_pwl")
+
+    def maxpool2d(self, x, y, ks, stride, pad, stream=None):
+        N, H, W, Cc = x.shape
+        _check(self._lib.nm_maxpool2d(self._h, _ptr(x), _ptr(y), dtype_of(x), N, H, W, Cc, ks, stride, pad,
+                                      _stream(stream)), "nm_maxpool2d")
+
+    def avgpool_global(self, x, y, stream=None):
+        N, H, W, Cc = x.shape
+        _check(self._lib.nm_avgpool_global(self._h, _ptr(x), _ptr(y), dtype_of(x), N, H, W, Cc, _stream(stream)),
+               "nm_avgpool_global")
+
+    @staticmethod
+    def resnet50_cfg(batch, dtype, num_classes=1000, relu_slot=SLOT_RELU, algo=ALGO_AUTO):
+        c = Resnet50Cfg()
+        c.batch, c.dtype, c.relu_slot, c.num_classes, c.algo = batch, dtype, relu_slot, num_classes, algo
+        return c
+
+    def resnet50_workspace_bytes(self, cfg) -> int:
+        return int(self._lib.nm_resnet50_workspace_bytes(C.byref(cfg)))
+
+    def resnet50_forward(self, conv_array, fc_w, fc_b, cfg, x, logits, workspace, stream=None):
+        _check(self._lib.nm_resnet50_forward(self._h, conv_array, _ptr(fc_w), _ptr(fc_b), C.byref(cfg), _ptr(x),
+                                             _ptr(logits), _ptr(workspace),
+                                             workspace.numel() * workspace.element_size(), _stream(stream)),
+               "nm_resnet50_forward")
+
+    def resnet50_forward_host(self, conv_array, fc_w, fc_b, cfg, x_host, logits_host, x_dev, logits_dev, workspace,
+                              stream=None):
+        _check(self._lib.nm_resnet50_forward_host(self._h, conv_array, _ptr(fc_w), _ptr(fc_b), C.byref(cfg),
+                                                  C.c_void_p(x_host.data_ptr()), C.c_void_p(logits_host.data_ptr()),
+                                                  _ptr(x_dev), _ptr(logits_dev), _ptr(workspace),
+                                                  workspace.numel() * workspace.element_size(), _stream(stream)),
+               "nm_resnet50_forward_host")
 
     # -- encoder ------------------------------------------------------------------
     @staticmethod

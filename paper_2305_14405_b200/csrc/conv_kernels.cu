@@ -1,0 +1,217 @@
+// CNN pieces of the PWL forward pass (Section 3.1: a convolution is a linear operator whose
+// matrix dimensions follow from width, height and channels; Section 3: ReLU is already
+// piecewise linear, here a 2-segment table in the GEMM epilogue).
+//
+// A convolution runs as out[M, Cout] = PWL(A[M, K] . W[Cout, K]^T + bias (+ residual)) with
+// M = N*Ho*Wo and K = kh*kw*Cin.  1x1 stride-1 convolutions use the NHWC activation as A
+// directly; every other shape first gathers A (im2col) into the caller's workspace, then
+// calls the same tensor-core linear kernel.  Max-pool and global average pool are small
+// bandwidth-bound kernels.
+#include "nm_common.cuh"
+
+namespace {
+
+// A[m][(ky*kw + kx)*Cin + c] = x[n][oy*s - p + ky][ox*s - p + kx][c], zero outside the image.
+// Vector path: Cin a multiple of 8, one 16-byte chunk per thread.
+template <typename T>
+__global__ void __launch_bounds__(256) im2col_vec_kernel(const T* __restrict__ x, T* __restrict__ A, int Nb, int H,
+                                                         int W, int Cin, int kh, int kw, int stride, int pad,
+                                                         int Ho, int Wo)
+{
+    const int c8n = Cin >> 3;
+    const int64_t chunks_per_row = (int64_t)kh * kw * c8n;
+    const int64_t total = (int64_t)Nb * Ho * Wo * chunks_per_row;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += step) {
+        const int64_t m = i / chunks_per_row;
+        const int r = (int)(i - m * chunks_per_row);
+        const int c8 = r % c8n;
+        const int kx = (r / c8n) % kw;
+        const int ky = r / (c8n * kw);
+        const int ox = (int)(m % Wo);
+        const int oy = (int)((m / Wo) % Ho);
+        const int n = (int)(m / ((int64_t)Wo * Ho));
+        const int iy = oy * stride - pad + ky, ix = ox * stride - pad + kx;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (iy >= 0 && iy < H && ix >= 0 && ix < W)
+            v = __ldg(reinterpret_cast<const uint4*>(x + (((int64_t)n * H + iy) * W + ix) * Cin + c8 * 8));
+        *reinterpret_cast<uint4*>(A + i * 8) = v;
+    }
+}
+
+// Scalar path (first layer, Cin = 3): rows padded with zeros to Kpad (a multiple of 8).
+template <typename T>
+__global__ void __launch_bounds__(256) im2col_scalar_kernel(const T* __restrict__ x, T* __restrict__ A, int Nb, int H,
+                                                            int W, int Cin, int kh, int kw, int stride, int pad,
+                                                            int Ho, int Wo, int Kpad)
+{
+    const int K = kh * kw * Cin;
+    const int64_t total = (int64_t)Nb * Ho * Wo * Kpad;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += step) {
+        const int64_t m = i / Kpad;
+        const int k = (int)(i - m * Kpad);
+        T v = NmType<T>::from_f(0.f);
+        if (k < K) {
+            const int c = k % Cin;
+            const int kx = (k / Cin) % kw;
+            const int ky = k / (Cin * kw);
+            const int ox = (int)(m % Wo);
+            const int oy = (int)((m / Wo) % Ho);
+            const int n = (int)(m / ((int64_t)Wo * Ho));
+            const int iy = oy * stride - pad + ky, ix = ox * stride - pad + kx;
+            if (iy >= 0 && iy < H && ix >= 0 && ix < W) v = x[(((int64_t)n * H + iy) * W + ix) * Cin + c];
+        }
+        A[i] = v;
+    }
+}
+
+// W[Cout][K] -> Wp[Cout][Kpad], zero padded
+template <typename T>
+__global__ void pad_rows_kernel(const T* __restrict__ w, T* __restrict__ wp, int rows, int K, int Kpad)
+{
+    const int64_t total = (int64_t)rows * Kpad;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / Kpad;
+        const int k = (int)(i - r * Kpad);
+        wp[i] = k < K ? w[r * K + k] : NmType<T>::from_f(0.f);
+    }
+}
+
+__device__ __forceinline__ float2 unpack2(__half2 v) { return __half22float2(v); }
+__device__ __forceinline__ float2 unpack2(__nv_bfloat162 v) { return __bfloat1622float2(v); }
+template <typename T> struct Vec2;
+template <> struct Vec2<__half> { using type = __half2; static __device__ __forceinline__ __half2 make(float a, float b) { return __floats2half2_rn(a, b); } };
+template <> struct Vec2<__nv_bfloat16> { using type = __nv_bfloat162; static __device__ __forceinline__ __nv_bfloat162 make(float a, float b) { return __floats2bfloat162_rn(a, b); } };
+
+// window maximum, padding cells ignored; 8 channels per thread
+template <typename T>
+__global__ void __launch_bounds__(256) maxpool_kernel(const T* __restrict__ x, T* __restrict__ y, int Nb, int H, int W,
+                                                      int C, int ks, int stride, int pad, int Ho, int Wo)
+{
+    using V2 = typename Vec2<T>::type;
+    const int c8n = C >> 3;
+    const int64_t total = (int64_t)Nb * Ho * Wo * c8n;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int c8 = (int)(i % c8n);
+        const int64_t m = i / c8n;
+        const int ox = (int)(m % Wo), oy = (int)((m / Wo) % Ho), n = (int)(m / ((int64_t)Wo * Ho));
+        float best[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) best[j] = -INFINITY;
+        for (int ky = 0; ky < ks; ++ky) {
+            const int iy = oy * stride - pad + ky;
+            if (iy < 0 || iy >= H) continue;
+            for (int kx = 0; kx < ks; ++kx) {
+                const int ix = ox * stride - pad + kx;
+                if (ix < 0 || ix >= W) continue;
+                const uint4 raw = __ldg(reinterpret_cast<const uint4*>(x + (((int64_t)n * H + iy) * W + ix) * C + c8 * 8));
+                const V2* h = reinterpret_cast<const V2*>(&raw);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 f = unpack2(h[j]);
+                    best[2 * j] = fmaxf(best[2 * j], f.x);
+                    best[2 * j + 1] = fmaxf(best[2 * j + 1], f.y);
+                }
+            }
+        }
+        uint4 out;
+        V2* o = reinterpret_cast<V2*>(&out);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[j] = Vec2<T>::make(best[2 * j], best[2 * j + 1]);
+        *reinterpret_cast<uint4*>(y + i * 8) = out;
+    }
+}
+
+// mean over the HW positions of each image: [N, HW, C] -> [N, C]; 8 channels per thread, fp32 sums
+template <typename T>
+__global__ void __launch_bounds__(256) avgpool_kernel(const T* __restrict__ x, T* __restrict__ y, int Nb, int HW, int C)
+{
+    using V2 = typename Vec2<T>::type;
+    const int c8n = C >> 3;
+    const int64_t total = (int64_t)Nb * c8n;
+    const float inv = 1.0f / (float)HW;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int c8 = (int)(i % c8n);
+        const int n = (int)(i / c8n);
+        float s[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s[j] = 0.f;
+        for (int p = 0; p < HW; ++p) {
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(x + ((int64_t)n * HW + p) * C + c8 * 8));
+            const V2* h = reinterpret_cast<const V2*>(&raw);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 f = unpack2(h[j]);
+                s[2 * j] += f.x;
+                s[2 * j + 1] += f.y;
+            }
+        }
+        uint4 out;
+        V2* o = reinterpret_cast<V2*>(&out);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[j] = Vec2<T>::make(s[2 * j] * inv, s[2 * j + 1] * inv);
+        *reinterpret_cast<uint4*>(y + ((int64_t)n * C + c8 * 8)) = out;
+    }
+}
+
+int grid_for(nm_ctx* ctx, int64_t total)
+{
+    int64_t want = (total + 255) / 256;
+    const int64_t cap = (int64_t)ctx->sm_count * 16;
+    return (int)(want < 1 ? 1 : (want > cap ? cap : want));
+}
+
+}  // namespace
+
+nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int Nb, int H, int W, int Cin, int kh,
+                           int kw, int stride, int pad, int Ho, int Wo, int Kpad, cudaStream_t st)
+{
+    const int64_t M = (int64_t)Nb * Ho * Wo;
+    NmLaunchScope scope(ctx, NM_KERNEL_IM2COL, (double)M * Kpad * 2.0 * nm_dtype_size(dt), st);
+    if (Cin % 8 == 0) {
+        const int64_t total = M * kh * kw * (Cin / 8);
+        if (dt == NM_F16)
+            im2col_vec_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)A, Nb, H, W, Cin, kh, kw, stride, pad, Ho, Wo);
+        else
+            im2col_vec_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)A, Nb, H, W, Cin, kh, kw, stride, pad, Ho, Wo);
+    } else {
+        const int64_t total = M * Kpad;
+        if (dt == NM_F16)
+            im2col_scalar_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)A, Nb, H, W, Cin, kh, kw, stride, pad, Ho, Wo, Kpad);
+        else
+            im2col_scalar_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)A, Nb, H, W, Cin, kh, kw, stride, pad, Ho, Wo, Kpad);
+    }
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+nm_status nm_launch_pad_rows(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, int rows, int K, int Kpad,
+                             cudaStream_t st)
+{
+    NmLaunchScope scope(ctx, NM_KERNEL_IM2COL, (double)rows * Kpad * 2.0 * nm_dtype_size(dt), st);
+    const int64_t total = (int64_t)rows * Kpad;
+    if (dt == NM_F16) pad_rows_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)w, (__half*)wp, rows, K, Kpad);
+    else pad_rows_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)wp, rows, K, Kpad);
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+nm_status nm_launch_maxpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int H, int W, int C, int ks,
+                            int stride, int pad, int Ho, int Wo, cudaStream_t st)
+{
+    const int64_t total = (int64_t)Nb * Ho * Wo * (C / 8);
+    NmLaunchScope scope(ctx, NM_KERNEL_POOL, ((double)Nb * H * W * C + (double)Nb * Ho * Wo * C) * nm_dtype_size(dt), st);
+    if (dt == NM_F16)
+        maxpool_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo);
+    else
+        maxpool_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo);
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+nm_status nm_launch_avgpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int HW, int C, cudaStream_t st)
+{
+    const int64_t total = (int64_t)Nb * (C / 8);
+    NmLaunchScope scope(ctx, NM_KERNEL_POOL, ((double)Nb * HW * C + (double)Nb * C) * nm_dtype_size(dt), st);
+    if (dt == NM_F16) avgpool_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)y, Nb, HW, C);
+    else avgpool_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, Nb, HW, C);
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}

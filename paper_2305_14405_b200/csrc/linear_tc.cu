@@ -42,6 +42,7 @@ struct TcArgs {
     int64_t M, N, K;
     const float* bias;
     int has_res;
+    int res_first;  // residual is added before the table instead of after
     const NmTable* tab;
     float a_scale;
     const float* w_scale;
@@ -427,6 +428,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             }
                         }
                     }
+                    if (has_res && a.res_first) add_res32<OutT>(&rsv[cc * WPC], v);
                     if (has_tab) {
                         if (a.idx_dump) {
 #pragma unroll
@@ -444,7 +446,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         for (int i = 0; i < 32; ++i)
                             if (row_ok && col0 + i < a.N) a.idx_dump[row * a.N + col0 + i] = -1;
                     }
-                    if (has_res) add_res32<OutT>(&rsv[cc * WPC], v);
+                    if (has_res && !a.res_first) add_res32<OutT>(&rsv[cc * WPC], v);
                     pack32<OutT>(v, &packed[cc * WPC], a.inv_out_scale);
                 }
                 // stage the group and send it: the previous store must have finished reading the buffer
@@ -519,6 +521,7 @@ nm_status launch(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
     a.M = d->M; a.N = d->N; a.K = d->K;
     a.bias = d->bias;
     a.has_res = d->residual ? 1 : 0;
+    a.res_first = d->res_first;
     a.tab = d->slot == NM_SLOT_NONE ? nullptr : ctx->d_tables + d->slot;
     a.n_seg = d->slot == NM_SLOT_NONE ? 0 : ctx->h_tables[d->slot].n;
     a.a_scale = d->a_scale; a.w_scale = d->w_scale; a.inv_out_scale = d->inv_out_scale;

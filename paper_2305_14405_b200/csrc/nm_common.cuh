@@ -542,3 +542,10 @@ bool nm_linear_tc_supported(const nm_linear_desc* d);
 nm_status nm_launch_attention_simt(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
 nm_status nm_launch_attention_tc(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
 bool nm_attention_tc_supported(const nm_attn_desc* d);
+nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int Nb, int H, int W, int Cin, int kh,
+                           int kw, int stride, int pad, int Ho, int Wo, int Kpad, cudaStream_t st);
+nm_status nm_launch_pad_rows(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, int rows, int K, int Kpad,
+                             cudaStream_t st);
+nm_status nm_launch_maxpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int H, int W, int C, int ks,
+                            int stride, int pad, int Ho, int Wo, cudaStream_t st);
+nm_status nm_launch_avgpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int HW, int C, cudaStream_t st);

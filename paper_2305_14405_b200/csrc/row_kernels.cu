@@ -79,60 +79,83 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restric
                                                         const float* __restrict__ beta, T* __restrict__ y,
                                                         int64_t rows, int H, float eps)
 {
+    // A warp walks over rows with a grid-wide stride; the raw 16-byte vectors of its NEXT row are
+    // already in flight while the current row is reduced and written, so every SM keeps several
+    // rows per warp outstanding instead of one short-lived row.
     constexpr int N = VecOf<T>::N;
     const int lane = threadIdx.x & 31;
-    const int warps_per_block = blockDim.x >> 5;
-    const int64_t row = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-    if (row >= rows) return;
-    const T* xr = x + row * H;
-    T* yr = y + row * H;
+    const int64_t warp0 = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int nvec = H / N;  // H is a multiple of N
-    float f[ITERS][N];
-    float sum = 0.f;
+    const float inv_h = tab->inv_h, off = tab->off, nm1 = (float)(tab->n - 1);
+    uint4 nxt[ITERS];
+    if (warp0 < rows) {
 #pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-        int v = it * 32 + lane;
-        if (v < nvec) {
-            load16<T>(xr + v * N, f[it]);
-#pragma unroll
-            for (int i = 0; i < N; ++i) sum += f[it][i];
+        for (int it = 0; it < ITERS; ++it) {
+            const int v = it * 32 + lane;
+            if (v < nvec) nxt[it] = *reinterpret_cast<const uint4*>(x + warp0 * H + v * N);
         }
     }
+    for (int64_t row = warp0; row < rows; row += nwarps) {
+        float f[ITERS][N];
+        float sum = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    const float mu = sum / (float)H;
-    float sq = 0.f;
+        for (int it = 0; it < ITERS; ++it) {
+            const int v = it * 32 + lane;
+            if (v < nvec) {
+                const T* e = reinterpret_cast<const T*>(&nxt[it]);
 #pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-        int v = it * 32 + lane;
-        if (v < nvec) {
-#pragma unroll
-            for (int i = 0; i < N; ++i) {
-                float dlt = f[it][i] - mu;
-                f[it][i] = dlt;
-                sq = __fmaf_rn(dlt, dlt, sq);
+                for (int i = 0; i < N; ++i) {
+                    f[it][i] = NmType<T>::to_f(e[i]);
+                    sum += f[it][i];
+                }
             }
         }
-    }
+        const int64_t nrow = row + nwarps;
+        if (nrow < rows) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-    const float var = sq / (float)H + eps;
-    const int s = nm_pwl_index(var, tab->inv_h, tab->off, (float)(tab->n - 1));
-    const float2 kb = tab->kb[s];
-    const float r = __fmaf_rn(kb.x, var, kb.y);
-#pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-        int v = it * 32 + lane;
-        if (v < nvec) {
-            float g[N], b[N];
-#pragma unroll
-            for (int i = 0; i < N; i += 4) {
-                *reinterpret_cast<float4*>(&g[i]) = __ldg(reinterpret_cast<const float4*>(gamma + v * N + i));
-                *reinterpret_cast<float4*>(&b[i]) = __ldg(reinterpret_cast<const float4*>(beta + v * N + i));
+            for (int it = 0; it < ITERS; ++it) {
+                const int v = it * 32 + lane;
+                if (v < nvec) nxt[it] = *reinterpret_cast<const uint4*>(x + nrow * H + v * N);
             }
+        }
 #pragma unroll
-            for (int i = 0; i < N; ++i) f[it][i] = __fmaf_rn(f[it][i] * r, g[i], b[i]);
-            store16<T>(yr + v * N, f[it]);
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float mu = sum / (float)H;
+        float sq = 0.f;
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            const int v = it * 32 + lane;
+            if (v < nvec) {
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+                    const float dlt = f[it][i] - mu;
+                    f[it][i] = dlt;
+                    sq = __fmaf_rn(dlt, dlt, sq);
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        const float var = sq / (float)H + eps;
+        const int s = nm_pwl_index(var, inv_h, off, nm1);
+        const float2 kb = tab->kb[s];
+        const float r = __fmaf_rn(kb.x, var, kb.y);
+        T* yr = y + row * H;
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            const int v = it * 32 + lane;
+            if (v < nvec) {
+                float g[N], b[N];
+#pragma unroll
+                for (int i = 0; i < N; i += 4) {
+                    *reinterpret_cast<float4*>(&g[i]) = __ldg(reinterpret_cast<const float4*>(gamma + v * N + i));
+                    *reinterpret_cast<float4*>(&b[i]) = __ldg(reinterpret_cast<const float4*>(beta + v * N + i));
+                }
+#pragma unroll
+                for (int i = 0; i < N; ++i) f[it][i] = __fmaf_rn(f[it][i] * r, g[i], b[i]);
+                store16<T>(yr + v * N, f[it]);
+            }
         }
     }
 }
@@ -170,8 +193,9 @@ nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const void* x, const float*
     const int nvec = H / N;
     const int iters = (nvec + 31) / 32;
     const int threads = 256;
-    const int64_t blocks = (rows + 7) / 8;
-    if (blocks > 0x7fffffffLL) return NM_ERR_SHAPE;
+    // a multiple of the SM count: 6 blocks of 8 warps per SM, each warp walking over rows
+    int64_t blocks = (rows + 7) / 8;
+    if (blocks > (int64_t)ctx->sm_count * 6) blocks = (int64_t)ctx->sm_count * 6;
  NmLaunchScope scope(ctx, NM_KERNEL_LAYERNORM, 2.0 * (double)rows * H * sizeof(T), st);
 #define NM_LN_CASE(I)                                                                                      \
     layernorm_kernel<T, I><<<(unsigned)blocks, threads, 0, st>>>(tab, (const T*)x, gamma, beta, (T*)y, rows, H, eps)

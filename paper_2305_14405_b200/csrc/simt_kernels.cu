@@ -22,6 +22,7 @@ struct LinArgs {
     int64_t M, N, K, lda, ldw, ldr, ldo;
     const float* bias;
     const void* residual;
+    int res_first;       // residual is added before the table instead of after
     const NmTable* tab;  // nullptr: no table
     float a_scale;
     const float* w_scale;
@@ -105,6 +106,7 @@ __global__ void __launch_bounds__(256) linear_simt_kernel(const InT* __restrict_
             } else {
                 x = acc[i][j] + bj;
             }
+            if (a.residual && a.res_first) x = x + load_res<OutT>((const OutT*)a.residual + gm * a.ldr + gn);
             int s = -1;
             if (a.tab) {
                 s = nm_pwl_index(x, inv_h, off, nm1);
@@ -112,7 +114,7 @@ __global__ void __launch_bounds__(256) linear_simt_kernel(const InT* __restrict_
                 x = __fmaf_rn(kb.x, x, kb.y);
             }
             if (a.idx_dump) a.idx_dump[gm * a.N + gn] = s;
-            if (a.residual) x = x + load_res<OutT>((const OutT*)a.residual + gm * a.ldr + gn);
+            if (a.residual && !a.res_first) x = x + load_res<OutT>((const OutT*)a.residual + gm * a.ldr + gn);
             store_out<OutT>(out + gm * a.ldo + gn, x, a.inv_out_scale);
         }
     }
@@ -190,7 +192,7 @@ nm_status launch_lin(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
 {
     LinArgs a;
     a.M = d->M; a.N = d->N; a.K = d->K; a.lda = d->lda; a.ldw = d->ldw; a.ldr = d->ldr; a.ldo = d->ldo;
-    a.bias = d->bias; a.residual = d->residual;
+    a.bias = d->bias; a.residual = d->residual; a.res_first = d->res_first;
     a.tab = d->slot == NM_SLOT_NONE ? nullptr : ctx->d_tables + d->slot;
     a.a_scale = d->a_scale; a.w_scale = d->w_scale; a.inv_out_scale = d->inv_out_scale;
     a.acc_dump = d->acc_dump; a.idx_dump = d->idx_dump;

@@ -1,0 +1,115 @@
+"""GPU parity, CNN path: convolution as GEMM with PWL (ReLU) epilogue, pooling, and the
+ResNet-50-shaped network against the oracle on seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs
+import nm_inputs_cnn
+import oracle
+import oracle.cnn
+from util import assert_close_bf16, load_tables_both, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx(nm):
+    c = nm.Context(0)
+    yield c
+    c.close()
+
+
+def relu_tables(ctx):
+    return load_tables_both(ctx, 2, {"relu": (-8.0, 8.0)})["relu"]
+
+
+@pytest.mark.parametrize("N,H,W,Cin,Cout,k,stride,pad", [
+    (2, 14, 14, 64, 128, 1, 1, 0),      # 1x1: activation used as the GEMM operand directly
+    (2, 14, 14, 64, 64, 3, 1, 1),       # 3x3 gather path
+    (3, 15, 13, 32, 72, 3, 2, 1),       # odd sizes, stride 2
+    (2, 28, 28, 256, 512, 1, 2, 0),     # strided 1x1 (projection shortcut)
+    (2, 40, 40, 3, 64, 7, 2, 3),        # first layer: Cin = 3, K = 147 padded to 152
+    (1, 9, 9, 16, 8, 5, 1, 2),
+])
+@pytest.mark.parametrize("epi", ["relu", "relu_res", "res_then_relu", "plain"])
+def test_conv2d_parity(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi):
+    relu = relu_tables(ctx)
+    rng = np.random.default_rng(N * 1000 + H + Cin + k)
+    x = nm_inputs.round_to(rng.standard_normal((N, H, W, Cin)).astype(np.float32), "f16")
+    w = nm_inputs.round_to((np.sqrt(2.0 / (Cin * k * k)) * rng.standard_normal((Cout, k, k, Cin))).astype(np.float32), "f16")
+    b = (0.1 * rng.standard_normal(Cout)).astype(np.float32)
+    Ho, Wo = (H + 2 * pad - k) // stride + 1, (W + 2 * pad - k) // stride + 1
+    res = nm_inputs.round_to(rng.standard_normal((N, Ho, Wo, Cout)).astype(np.float32), "f16") if "res" in epi else None
+    xd = torch.from_numpy(x).cuda().half()
+    wd = torch.from_numpy(w).cuda().half()
+    out = torch.full((N, Ho, Wo, Cout), float("nan"), dtype=torch.float16, device="cuda")
+    bd = torch.from_numpy(b).cuda()                      # the descriptor holds raw pointers: keep the tensors alive
+    rd = torch.from_numpy(res).cuda().half() if res is not None else None
+    d = nm.Context.conv_desc(xd, wd, out, stride, pad, bias=bd, residual=rd,
+                             slot=nm.SLOT_NONE if epi == "plain" else nm.SLOT_RELU, res_first=(epi == "res_then_relu"))
+    ws_bytes = ctx.conv2d_workspace_bytes(d)
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
+    ctx.conv2d_pwl(d, ws)
+    ctx.check_device_status()
+    if epi == "res_then_relu":
+        ref = oracle.pwl_eval(relu, oracle.conv2d_nhwc(x, w, stride, pad, b, res, None))[0]
+    else:
+        ref = oracle.conv2d_nhwc(x, w, stride, pad, b, res, None if epi == "plain" else relu)
+    assert_close_bf16(to_np(out), ref, "conv %s" % epi)
+
+
+def test_pools_parity(nm, ctx):
+    rng = np.random.default_rng(5)
+    x = nm_inputs.round_to(rng.standard_normal((3, 23, 17, 64)).astype(np.float32), "f16")
+    xd = torch.from_numpy(x).cuda().half()
+    y = torch.empty((3, 12, 9, 64), dtype=torch.float16, device="cuda")
+    ctx.maxpool2d(xd, y, 3, 2, 1)
+    assert np.array_equal(to_np(y), oracle.maxpool_nhwc(x, 3, 2, 1))          # a maximum of fp16 values: exact
+    a = torch.empty((3, 64), dtype=torch.float16, device="cuda")
+    ctx.avgpool_global(xd, a)
+    assert_close_bf16(to_np(a), oracle.avgpool_nhwc(x), "avgpool")
+    with pytest.raises(nm.NmError) as ei:
+        ctx.maxpool2d(xd[..., :12].contiguous(), y, 3, 2, 1)                  # channels not a multiple of 8
+    assert ei.value.code == 2
+
+
+@pytest.mark.parametrize("random_bn", [False, True])
+def test_resnet50_two_images(nm, ctx, random_bn):
+    """The whole ResNet-50-shaped network (53 convolutions, pools, classifier) on two 224x224 images,
+    fp16 NHWC, BatchNorm folded into the convolutions, against the fp64 oracle."""
+    from paper_2305_14405_b200.harness_cnn import Resnet50Model
+    relu = relu_tables(ctx)
+    x, convs, fc_w, fc_b = nm_inputs_cnn.resnet50_inputs(2, seed=0, random_bn=random_bn)
+    m = Resnet50Model(ctx, 2, convs, fc_w, fc_b)
+    logits = m.forward(torch.from_numpy(x).cuda().half())
+    ctx.check_device_status()
+    ref = oracle.cnn.resnet50(x, convs, fc_w, fc_b, relu)
+    got = to_np(logits)
+    err = np.abs(got - ref)
+    rms = np.sqrt((ref ** 2).mean())
+    print("resnet50 logits: max |ref| %.3f, rms ref %.3f, max err %.4f, rms err %.5f"
+          % (np.abs(ref).max(), rms, err.max(), np.sqrt((err ** 2).mean())))
+    # A logit is a sum of 2048 products of magnitude up to ~1e3 that largely cancel: its rounding error
+    # scales with the typical logit magnitude, not with its own value, so elements near zero are held to
+    # the bound of an rms-sized element (the same rule as for the fp32 path, at the fp16 tolerance).
+    bound = 1e-2 + 1e-2 * np.maximum(np.abs(ref), rms)
+    assert np.all(np.isfinite(got)) and not (err > bound).any(), "%d outside" % (err > bound).sum()
+
+
+def test_resnet50_full_batch_sampled_images(nm, ctx):
+    """Config 5 in the benchmark's launch configuration (batch 128, fp16 NHWC, random folded BatchNorm):
+    images are independent, so the oracle runs two sampled images through the whole network."""
+    from paper_2305_14405_b200.harness_cnn import Resnet50Model
+    relu = relu_tables(ctx)
+    x, convs, fc_w, fc_b = nm_inputs_cnn.resnet50_inputs(128, seed=0, random_bn=True)
+    m = Resnet50Model(ctx, 128, convs, fc_w, fc_b)
+    logits = m.forward(torch.from_numpy(x).cuda().half())
+    ctx.check_device_status()
+    got_all = to_np(logits)
+    assert np.all(np.isfinite(got_all))
+    for i in (5, 127):
+        ref = oracle.cnn.resnet50(x[i:i + 1], convs, fc_w, fc_b, relu)
+        rms = np.sqrt((ref ** 2).mean())
+        err = np.abs(got_all[i:i + 1] - ref)
+        assert not (err > 1e-2 + 1e-2 * np.maximum(np.abs(ref), rms)).any(), "image %d: max err %.3f" % (i, err.max())

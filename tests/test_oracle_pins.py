@@ -496,3 +496,33 @@ def test_int8_encoder_layer_against_library_routines():
     # a code on a rounding boundary may differ between two fp64 summation orders: allow a few elements
     err = np.abs(got - ref)
     assert (err > 1e-9).mean() < 0.02 and np.median(err) < 1e-12
+
+
+def test_resnet50_composition_against_torch():
+    """The oracle's ResNet-50-shaped network (a composition of its own conv / pool / linear routines)
+    against torch.nn.functional in fp64 on a reduced image: pins the block wiring (projection shortcut
+    only in a stage's first block, stride in the 3x3, ReLU after the add) and the folded-BatchNorm inputs."""
+    import nm_inputs_cnn
+    import oracle.cnn
+    F = torch.nn.functional
+    x, convs, fc_w, fc_b = nm_inputs_cnn.resnet50_inputs(1, seed=3, random_bn=True, image=64, num_classes=16)
+    relu = Table.secant(oracle.RELU, 2, -8.0, 8.0)
+    got = oracle.cnn.resnet50(x, convs, fc_w, fc_b, relu)
+
+    def conv(inp, c):
+        _, _, _, s, p = c["spec"]
+        return F.conv2d(inp, torch.from_numpy(c["w"].astype(np.float64)).permute(0, 3, 1, 2),
+                        torch.from_numpy(c["b"].astype(np.float64)), stride=s, padding=p)
+
+    it = iter(convs)
+    y = torch.from_numpy(x.astype(np.float64)).permute(0, 3, 1, 2)
+    y = F.max_pool2d(F.relu(conv(y, next(it))), 3, 2, 1)
+    for nb in (3, 4, 6, 3):
+        for b in range(nb):
+            ca, cb, cc = next(it), next(it), next(it)
+            t = F.relu(conv(F.relu(conv(y, ca)), cb))
+            sc = conv(y, next(it)) if b == 0 else y
+            y = F.relu(conv(t, cc) + sc)
+    ref = (y.mean(dim=(2, 3)) @ torch.from_numpy(fc_w.astype(np.float64)).T + torch.from_numpy(fc_b.astype(np.float64))).numpy()
+    assert np.allclose(got, ref, rtol=1e-10, atol=1e-9)
+    assert len(convs) == 53 and sum(c["w"].size for c in convs) + fc_w.size > 23e6   # ResNet-50's ~23.5 M conv weights
