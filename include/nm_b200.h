@@ -84,6 +84,22 @@ nm_status nm_ctx_poll_status(nm_ctx* ctx, int* device_status, void* stream);
  * k_host, b_host: host arrays of n floats, written.  1 <= n <= NM_MAX_SEGMENTS. */
 nm_status nm_pwl_table_build(int func, int n, float x_min, float x_max, float* k_host, float* b_host);
 
+/* Host-only construction of an ELASTIC table (Section 3.2: Algorithm 1 without its training loop):
+ * Algorithm 2 "Horizontal Size Optimization" walks [r_min, r_max] in primary segments of length dLx
+ * and opens a new segment only where the primary slope differs from the slope remembered at the last
+ * kept start point by more than dK_th; Algorithm 3 "Vertical Bias Correction" gives each segment its
+ * secant k, b and, when bias_correct != 0, shifts b by dE = mean of func over the segment minus the mean
+ * of the secant, if |dE| > e_th (the reading of the section's prose).
+ * The result is returned on the PRIMARY grid: n_cells = (r_max - r_min)/dLx equal cells (at most
+ * NM_MAX_SEGMENTS; the range must be a whole number of primary segments), every cell carrying the k, b of
+ * the merged segment it belongs to, so the table loads with nm_pwl_table_load(slot, n_cells, r_min, r_max,
+ * k, b) and the kernels evaluate it with the same one-FMA index as any other table.  *n_segments_out is
+ * the number of distinct segments Algorithm 2 kept (the parameter count the paper reports on).
+ * k_host, b_host: host arrays of NM_MAX_SEGMENTS floats. */
+nm_status nm_pwl_table_build_elastic(int func, float r_min, float r_max, float dLx, float dK_th, int bias_correct,
+                                     float e_th, int* n_cells_out, int* n_segments_out, float* k_host,
+                                     float* b_host);
+
 /* Copies a table into `slot` ("parameters k and b of each segment are pre-stored
  * ... and indexed by the segment number", Section 3.2).  The table has n equal
  * segments on [x_min, x_max]; k_host/b_host are host arrays of n floats and may

@@ -28,7 +28,7 @@ EXPORTS = [
     "nm_layernorm_pwl", "nm_quantize_i8", "nm_encoder_workspace_bytes", "nm_encoder_layer", "nm_encoder_stack",
     "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
     "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
-    "nm_resnet50_forward", "nm_resnet50_forward_host",
+    "nm_resnet50_forward", "nm_resnet50_forward_host", "nm_pwl_table_build_elastic",
 ]
 KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc",
                 "im2col", "pool")
@@ -108,6 +108,9 @@ def load():
     lib.nm_ctx_launch_count.argtypes = [C.c_void_p, C.c_int]
     lib.nm_pwl_table_build.argtypes = [C.c_int, C.c_int, C.c_float, C.c_float, C.POINTER(C.c_float),
                                        C.POINTER(C.c_float)]
+    lib.nm_pwl_table_build_elastic.argtypes = [C.c_int, C.c_float, C.c_float, C.c_float, C.c_float, C.c_int, C.c_float,
+                                               C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_float),
+                                               C.POINTER(C.c_float)]
     lib.nm_pwl_table_load.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.POINTER(C.c_float),
                                       C.POINTER(C.c_float)]
     lib.nm_pwl_apply.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
@@ -183,6 +186,16 @@ def pwl_table_build(func: int, n: int, x_min: float, x_max: float):
     b = (C.c_float * n)()
     _check(load().nm_pwl_table_build(func, n, x_min, x_max, k, b), "nm_pwl_table_build")
     return list(k), list(b)
+
+
+def pwl_table_build_elastic(func, r_min, r_max, dLx, dK_th, bias_correct=True, e_th=0.0):
+    """nm_pwl_table_build_elastic (Algorithms 2 and 3): returns (n_cells, k, b, n_segments) on the primary grid."""
+    k = (C.c_float * 256)()
+    b = (C.c_float * 256)()
+    n, nseg = C.c_int(0), C.c_int(0)
+    _check(load().nm_pwl_table_build_elastic(func, r_min, r_max, dLx, dK_th, 1 if bias_correct else 0, e_th,
+                                             C.byref(n), C.byref(nseg), k, b), "nm_pwl_table_build_elastic")
+    return n.value, list(k)[:n.value], list(b)[:n.value], nseg.value
 
 
 class Context:

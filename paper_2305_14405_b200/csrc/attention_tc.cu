@@ -40,22 +40,7 @@ struct AttnArgs {
     int nbuf;    // P buffers
     int p_in_k;  // P buffers reuse the K tile region (L >= 256)
     uint32_t tmem_cols, o_col;
-#ifdef NM_EXP_TIMELINE
-    long long* dbg;  // development only: per-CTA timestamps
-#endif
 };
-#ifdef NM_EXP_TIMELINE
-#include <stdlib.h>
-__device__ __forceinline__ long long nm_gtime_a()
-{
-    long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define NM_TLA(slot) do { if (a.dbg && blockIdx.x < 4) a.dbg[blockIdx.x * 64 + (slot)] = nm_gtime_a(); } while (0)
-#else
-#define NM_TLA(slot) do {} while (0)
-#endif
 
 template <typename T> struct AttnT;
 template <> struct AttnT<__nv_bfloat16> {
@@ -132,7 +117,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int b = blockIdx.x / (blocks_per_seq * a.heads);
 
     if (threadIdx.x == 0) {
-        NM_TLA(0);
         abort_flag = 0;
         nm_prefetch_tmap(&tmQ);
         nm_prefetch_tmap(&tmK);
@@ -174,10 +158,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             nm_mbar_expect_tx(&bar_v, (uint32_t)(L * ROWB));
             for (int j = 0; j < L / 128; ++j) nm_tma_load_3d(v_s + (size_t)j * 128 * ROWB, &tmV, g * HD, j * 128, b, &bar_v);
             // ---- S = Q K^T, 128 keys per instruction group
-            NM_TLA(1);
             ok = nm_mbar_wait(&bar_qk, 0, abortp, a.status);
             if (ok) {
-                NM_TLA(2);
                 nm_tc_fence_after();
                 const uint64_t qdesc = nm_smem_desc_sw128(nm_smem_u32(q_s));
                 for (int jc = 0; jc < L / 128; ++jc) {
@@ -187,7 +169,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         nm_mma_f16(tmem_base + (uint32_t)(jc * 128), qdesc + 2 * k, kdesc + 2 * k, IDESC_QK, k != 0);
                 }
                 nm_tc_commit(&bar_s);
-                NM_TLA(3);
                 ok = nm_mbar_wait(&bar_v, 0, abortp, a.status);
             }
             // ---- O += P V, 64 keys per P buffer
@@ -195,7 +176,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int buf = c % a.nbuf;
                 ok = nm_mbar_wait(&bar_p_full[buf], (uint32_t)((c / a.nbuf) & 1), abortp, a.status);
                 if (!ok) break;
-                NM_TLA(20 + c);
                 nm_tc_fence_after();
                 const uint64_t pdesc = nm_smem_desc_sw128(nm_smem_u32(p_s + (size_t)buf * BQ * ROWB));
 #pragma unroll
@@ -205,10 +185,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     nm_mma_f16(tmem_base + a.o_col, pdesc + 2 * k, vdesc, IDESC_PV, (c | k) != 0);
                 }
                 nm_tc_commit(&bar_p_empty[buf]);
-                NM_TLA(30 + c);
             }
             if (ok) nm_tc_commit(&bar_o);
-            NM_TLA(4);
             if (!ok) {
                 // bounded drain: pending copies and MMAs get time to finish before teardown
                 long long t0 = clock64();
@@ -230,7 +208,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_s, 0, abortp, a.status) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
         float m = -INFINITY;
-        if (warp == 1 && lane == 0) NM_TLA(8);
         if (ok) {
             (void)nm_mbar_try_wait(&bar_s, 0);
             nm_tc_fence_after();
@@ -251,13 +228,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 m = max3(m, m0, m1);
             }
         }
-        if (warp == 1 && lane == 0) NM_TLA(9);
         s_red[h][row] = m;
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
 #pragma unroll
         for (int i = 0; i < NH; ++i) m = fmaxf(m, s_red[i][row]);  // the FINAL row maximum
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-        if (warp == 1 && lane == 0) NM_TLA(10);
         const float neg_ms = -(m * a.scale);
         float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
         if (ok) {
@@ -309,7 +284,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 __syncwarp();
             }
         }
-        if (warp == 1 && lane == 0) NM_TLA(11);
         s_red[h][row] = (sum0 + sum1) + (sum2 + sum3);
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
         float sum = 0.f;
@@ -323,7 +297,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_o, 0, abortp, a.status) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (ok) {
-                if (warp == 1 && lane == 0) NM_TLA(12);
                 (void)nm_mbar_try_wait(&bar_o, 0);
                 nm_tc_fence_after();
                 constexpr int CH = HD / NH;  // channels per warp group: 16 or 32
@@ -346,7 +319,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     nm_tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) NM_TLA(13);
     if (warp == 0) {
         __syncwarp();
         nm_tc_fence_after();
@@ -383,9 +355,6 @@ nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
     a.out = d->out;
     a.status = ctx->d_status;
     a.n_exp = ctx->h_tables[d->exp_slot].n;
-#ifdef NM_EXP_TIMELINE
-    a.dbg = getenv("NM_DBG_PTR") ? (long long*)strtoull(getenv("NM_DBG_PTR"), nullptr, 16) : nullptr;
-#endif
     const int L = d->L;
     a.p_in_k = L >= 256 ? 1 : 0;
     a.nbuf = L >= 256 ? L / 128 : 2;

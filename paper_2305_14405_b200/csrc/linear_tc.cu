@@ -51,22 +51,7 @@ struct TcArgs {
     int32_t* idx_dump;
     int* status;
     int num_n_tiles, num_tiles, num_k_blocks, stages, n_seg;
-#ifdef NM_EXP_TIMELINE
-    long long* dbg;  // development only: per-CTA timestamps
-#endif
 };
-#ifdef NM_EXP_TIMELINE
-#include <stdlib.h>
-__device__ __forceinline__ long long nm_gtime()
-{
-    long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define NM_TL(slot) do { if (a.dbg && blockIdx.x < 8) a.dbg[blockIdx.x * 64 + (slot)] = nm_gtime(); } while (0)
-#else
-#define NM_TL(slot) do {} while (0)
-#endif
 
 template <typename InT> struct TcIn;
 template <> struct TcIn<__nv_bfloat16> {
@@ -184,7 +169,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int tile_step = TWO ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
-        NM_TL(0);
         abort_flag = 0;
         nm_prefetch_tmap(&tmA);
         nm_prefetch_tmap(&tmW);
@@ -218,8 +202,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     nm_tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_flag;
-    if (threadIdx.x == 0) NM_TL(1);
-    int tl_tile = 0;
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -232,7 +214,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int n0 = (tile % a.num_n_tiles) * BN + (int)rank * B_ROWS;
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
                     if (!nm_mbar_wait(&bar_empty[stage], phase ^ 1u, abortp, a.status)) { ok = false; break; }
-                    if (kb == 0 && tl_tile < 4) { NM_TL(4 + tl_tile); ++tl_tile; }
                     uint8_t* sa = tiles + (size_t)stage * STAGE_BYTES;
                     if constexpr (TWO) {
                         // both CTAs' copies are counted on the leader's barrier
@@ -265,11 +246,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!(TWO ? nm_mbar_wait_cluster(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status)
                           : nm_mbar_wait(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status))) { ok = false; break; }
                 nm_tc_fence_after();
-                if (tl_tile < 4) NM_TL(8 + tl_tile);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
                     if (!nm_mbar_wait(&bar_full[stage], phase, abortp, a.status)) { ok = false; break; }
-                    if (kb == 0 && tl_tile < 4) NM_TL(12 + tl_tile);
                     nm_tc_fence_after();
                     const uint32_t sa = nm_smem_u32(tiles + (size_t)stage * STAGE_BYTES);
                     const uint64_t adesc = nm_smem_desc_sw128(sa);
@@ -293,7 +272,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!ok) break;
                 if constexpr (TWO) nm_tc_commit2(&bar_acc_full[buf], 3);
                 else nm_tc_commit(&bar_acc_full[buf]);
-                if (tl_tile < 4) { NM_TL(16 + tl_tile); ++tl_tile; }
                 buf ^= 1;
                 if (buf == 0) acc_phase ^= 1u;
             }
@@ -338,7 +316,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (!ok) break;
             (void)nm_mbar_try_wait(&bar_acc_full[buf], acc_phase);  // every lane observes the phase itself
             nm_tc_fence_after();
-            if (warp == 2 && lane == 0 && tl_tile < 4) NM_TL(20 + tl_tile);
             const int64_t row = (int64_t)m0 + q * 32 + lane;
             const bool row_ok = row < a.M;
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2));
@@ -465,7 +442,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (lane == 0 && ok && n0 + g * GROUP_COLS < a.N && m0 + q * 32 < a.M)
                     nm_tma_store_2d(&tmO, my_out, n0 + g * GROUP_COLS, m0 + q * 32);
             }
-            if (warp == 2 && lane == 0 && tl_tile < 4) { NM_TL(24 + tl_tile); ++tl_tile; }
             buf ^= 1;
             if (buf == 0) acc_phase ^= 1u;
         }
@@ -476,7 +452,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ---------------------------------------------------- teardown (all paths)
     nm_tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) NM_TL(2);
     if constexpr (TWO) nm_cluster_sync();  // the peer may still use barriers / tensor memory of the pair
     if (warp == 1) {
         __syncwarp();
@@ -527,9 +502,6 @@ nm_status launch(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
     a.a_scale = d->a_scale; a.w_scale = d->w_scale; a.inv_out_scale = d->inv_out_scale;
     a.acc_dump = d->acc_dump; a.idx_dump = d->idx_dump;
     a.status = ctx->d_status;
-#ifdef NM_EXP_TIMELINE
-    a.dbg = getenv("NM_DBG_PTR") ? (long long*)strtoull(getenv("NM_DBG_PTR"), nullptr, 16) : nullptr;
-#endif
     const int bk = ROW_BYTES / (int)sizeof(InT);
     const int64_t m_tiles = (d->M + TILE_M - 1) / TILE_M;
     a.num_n_tiles = (int)((d->N + BN - 1) / BN);

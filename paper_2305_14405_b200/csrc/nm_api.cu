@@ -33,6 +33,25 @@ double exact_fn(int func, double x)
     return NAN;
 }
 
+// F with F' = f, for the segment mean of Algorithm 3
+double antiderivative_fn(int func, double x)
+{
+    switch (func) {
+    case NM_FUNC_GELU: {
+        const double Phi = 0.5 * (1.0 + erf(x / sqrt(2.0)));
+        const double phi = exp(-0.5 * x * x) / sqrt(2.0 * 3.14159265358979323846);
+        return 0.5 * (x * x - 1.0) * Phi + 0.5 * x * phi;
+    }
+    case NM_FUNC_EXP: return exp(x);
+    case NM_FUNC_RECIP: return log(x);
+    case NM_FUNC_RSQRT: return 2.0 * sqrt(x);
+    case NM_FUNC_RELU: return x > 0.0 ? 0.5 * x * x : 0.0;
+    case NM_FUNC_SQRT: return (2.0 / 3.0) * x * sqrt(x);
+    case NM_FUNC_IDENTITY: return 0.5 * x * x;
+    }
+    return NAN;
+}
+
 }  // namespace
 
 extern "C" {
@@ -165,6 +184,54 @@ nm_status nm_pwl_table_build(int func, int n, float x_min, float x_max, float* k
         k_host[i] = (float)k;
         b_host[i] = (float)(f0 - k * x0);
     }
+    return NM_OK;
+}
+
+nm_status nm_pwl_table_build_elastic(int func, float r_min, float r_max, float dLx, float dK_th, int bias_correct,
+                                     float e_th, int* n_cells_out, int* n_segments_out, float* k_host, float* b_host)
+{
+    if (!n_cells_out || !n_segments_out || !k_host || !b_host) return NM_ERR_INVALID_ARG;
+    if (func < NM_FUNC_GELU || func > NM_FUNC_IDENTITY) return NM_ERR_INVALID_ARG;
+    if (!(r_max > r_min) || !(dLx > 0.f) || dK_th < 0.f || e_th < 0.f) return NM_ERR_SHAPE;
+    const double lo = (double)r_min, hi = (double)r_max, step = (double)dLx;
+    const double cells = (hi - lo) / step;
+    const int n = (int)llround(cells);
+    if (n < 1 || n > NM_MAX_SEGMENTS || fabs(cells - (double)n) > 1e-6 * cells) return NM_ERR_SHAPE;
+    // Algorithm 2: start cells of the kept segments
+    int start[NM_MAX_SEGMENTS + 1];
+    int nseg = 0;
+    start[nseg++] = 0;
+    auto cell_slope = [&](int c) {
+        const double x0 = lo + (double)c * step, x1 = lo + (double)(c + 1) * step;
+        return (exact_fn(func, x1) - exact_fn(func, x0)) / step;
+    };
+    double kref = cell_slope(0);
+    for (int c = 1; c < n; ++c) {
+        const double kc = cell_slope(c);
+        if (fabs(kc - kref) > (double)dK_th) {
+            start[nseg++] = c;
+            kref = kc;
+        }
+    }
+    start[nseg] = n;
+    // Algorithm 3 per kept segment, replicated over its primary cells
+    for (int s = 0; s < nseg; ++s) {
+        const double xa = lo + (double)start[s] * step;
+        const double xb = (start[s + 1] == n) ? hi : lo + (double)start[s + 1] * step;
+        const double fa = exact_fn(func, xa), fb = exact_fn(func, xb);
+        const double k = (fb - fa) / (xb - xa);
+        double b = fa - k * xa;
+        if (bias_correct) {
+            const double dE = (antiderivative_fn(func, xb) - antiderivative_fn(func, xa)) / (xb - xa) - 0.5 * (fa + fb);
+            if (fabs(dE) > (double)e_th) b += dE;
+        }
+        for (int c = start[s]; c < start[s + 1]; ++c) {
+            k_host[c] = (float)k;
+            b_host[c] = (float)b;
+        }
+    }
+    *n_cells_out = n;
+    *n_segments_out = nseg;
     return NM_OK;
 }
 

@@ -113,3 +113,29 @@ def test_quantize_bit_exact(nm, ctx, dtype):
     q = torch.empty(x.size, dtype=torch.int8, device="cuda")
     ctx.quantize_i8(xd, inv, q)
     assert np.array_equal(q.cpu().numpy(), oracle.quantize_i8(x, scale))
+
+
+@pytest.mark.parametrize("func,lo,hi,dLx,dK", [("gelu", -4.0, 4.0, 0.125, 0.02), ("exp", -8.0, 0.0, 0.125, 0.01),
+                                               ("recip", 1.0, 33.0, 0.25, 0.002)])
+def test_elastic_tables_evaluate_bit_exact(nm, ctx, func, lo, hi, dLx, dK):
+    """Tables with Algorithm 2's merged segments and Algorithm 3's bias correction (not continuous any
+    more: the fp32 index contract decides which side of a jump an input lands on) evaluate bit for bit."""
+    from util import FUNCS, oracle_elastic_table
+    n, k, b, nseg = nm.pwl_table_build_elastic(FUNCS[func], lo, hi, dLx, dK, bias_correct=True)
+    t, _ = oracle_elastic_table(FUNCS[func], lo, hi, dLx, dK, bias_correct=True)
+    assert nseg < n
+    ctx.pwl_table_load(nm.SLOT_USER0, n, lo, hi, k, b)
+    x = nm_inputs.pwl_probe_points(lo, hi, n, 50021, seed=7)
+    x = x[np.isfinite(x)]
+    xd = torch.from_numpy(x).cuda()
+    yd = torch.empty_like(xd)
+    idx = torch.empty(x.size, dtype=torch.int32, device="cuda")
+    ctx.pwl_apply(nm.SLOT_USER0, xd, yd, idx)
+    y_ref, idx_ref = oracle.pwl_eval_f32(t, x)
+    assert np.array_equal(idx.cpu().numpy(), idx_ref)
+    assert np.array_equal(yd.cpu().numpy().view(np.uint32), y_ref.view(np.uint32))
+    # and the elastic table approximates the function at least as well (in mean square) as its secants
+    xx = np.linspace(lo, hi, 20001)[1:-1]
+    exact = oracle.exact(FUNCS[func], xx)
+    t0, _ = oracle_elastic_table(FUNCS[func], lo, hi, dLx, dK, bias_correct=False)
+    assert ((t(xx) - exact) ** 2).mean() < ((t0(xx) - exact) ** 2).mean()

@@ -74,3 +74,27 @@ def test_product_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in src and "from oracle" not in src and "nm_oracle" not in src, f
+
+
+@pytest.mark.parametrize("func,lo,hi,dLx,dK", [(nm.FUNC_GELU, -4.0, 4.0, 0.5, 0.1), (nm.FUNC_GELU, -4.0, 4.0, 0.125, 0.02),
+                                               (nm.FUNC_EXP, -8.0, 0.0, 0.125, 0.01), (nm.FUNC_RECIP, 1.0, 33.0, 0.25, 0.002),
+                                               (nm.FUNC_SQRT, 0.25, 8.25, 0.0625, 0.01), (nm.FUNC_RSQRT, 0.25, 4.25, 0.03125, 0.02)])
+@pytest.mark.parametrize("bias", [False, True])
+def test_elastic_table_builder_matches_oracle_bitwise(lib, func, lo, hi, dLx, dK, bias):
+    """Algorithms 2 and 3 in the library's host code against the oracle's (pinned) routines."""
+    from util import oracle_elastic_table
+    n, k, b, nseg = nm.pwl_table_build_elastic(func, lo, hi, dLx, dK, bias_correct=bias)
+    t, nseg_ref = oracle_elastic_table(func, lo, hi, dLx, dK, bias_correct=bias)
+    assert n == t.n and nseg == nseg_ref and nseg < n          # segments were merged
+    assert np.array_equal(np.asarray(k, np.float32), t.k)
+    assert np.array_equal(np.asarray(b, np.float32), t.b)
+
+
+def test_elastic_table_builder_rejects_bad_requests(lib):
+    k = (C.c_float * 256)()
+    n, s = C.c_int(0), C.c_int(0)
+    f = lib.nm_pwl_table_build_elastic
+    assert f(0, -4.0, 4.0, 0.01, 0.1, 1, 0.0, C.byref(n), C.byref(s), k, k) == 2     # 800 primary cells > 256
+    assert f(0, -4.0, 4.0, 0.3, 0.1, 1, 0.0, C.byref(n), C.byref(s), k, k) == 2      # range not a whole number of cells
+    assert f(0, 4.0, -4.0, 0.5, 0.1, 1, 0.0, C.byref(n), C.byref(s), k, k) == 2
+    assert f(9, -4.0, 4.0, 0.5, 0.1, 1, 0.0, C.byref(n), C.byref(s), k, k) == 1

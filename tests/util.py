@@ -54,3 +54,18 @@ def load_tables_both(ctx, n, ranges):
         assert np.array_equal(np.asarray(b, np.float32), t.b), name
         out[name] = t
     return out
+
+
+def oracle_elastic_table(func, r_min, r_max, dLx, dK_th, bias_correct=True, e_th=0.0):
+    """The elastic table (Algorithm 2 start points, Algorithm 3 parameters) built from the oracle's own
+    routines and laid on the primary grid: returns (oracle.Table on n_cells equal cells, n_segments)."""
+    import oracle
+    starts = oracle.hsize_startpoints(func, dLx, dK_th, r_min, r_max)
+    xs = np.concatenate([starts, [r_max]])
+    k, b = oracle.secant_points(func, xs)
+    if bias_correct:
+        b, _ = oracle.bias_correct(func, xs, b, e_th)
+    n_cells = int(round((r_max - r_min) / dLx))
+    cell_x = r_min + dLx * np.arange(n_cells)
+    seg = np.searchsorted(starts, cell_x + 1e-9 * dLx, side="right") - 1
+    return oracle.Table(n_cells, r_min, r_max, k[seg].astype(np.float32), b[seg].astype(np.float32)), len(starts)
