@@ -348,6 +348,13 @@ nm_status nm_resnet50_forward_host(nm_ctx* ctx, const nm_conv_params* convs, con
 nm_status nm_encoder_layer_static(nm_ctx* ctx, const nm_encoder_weights* w, const nm_encoder_cfg* cfg,
                                   const void* x, void* y, void* stream);
 
+/* Diagnostic for the failure-detection path (no counterpart in the paper): launches a one-warp kernel
+ * that waits on a barrier nothing ever arrives on.  Like every wait in the tensor-core kernels, the
+ * wait is bounded: after limit_cycles SM clock cycles (1 .. 4e9) it gives up, writes NM_ERR_TIMEOUT to
+ * the context's status word and the kernel returns normally, leaving the context usable.
+ * nm_ctx_poll_status then reports NM_ERR_TIMEOUT. */
+nm_status nm_selftest_bounded_wait(nm_ctx* ctx, int64_t limit_cycles, void* stream);
+
 /* Number of kernels the library has launched through this context since creation
  * (or since the last call with reset != 0). */
 int64_t nm_ctx_launch_count(nm_ctx* ctx, int reset);

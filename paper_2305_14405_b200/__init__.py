@@ -29,6 +29,7 @@ EXPORTS = [
     "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
     "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
     "nm_resnet50_forward", "nm_resnet50_forward_host", "nm_pwl_table_build_elastic",
+    "nm_selftest_bounded_wait",
 ]
 KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc",
                 "im2col", "pool")
@@ -144,6 +145,7 @@ def load():
     lib.nm_resnet50_forward_host.argtypes = [C.c_void_p, C.POINTER(ConvParams), C.c_void_p, C.c_void_p,
                                              C.POINTER(Resnet50Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.nm_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.nm_ctx_profile_enable.argtypes = [C.c_void_p, C.c_int]
     lib.nm_ctx_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_double),
                                         C.POINTER(C.c_double)]
@@ -247,6 +249,10 @@ class Context:
         v = self.poll_status(stream)
         if v != NM_OK:
             raise NmError(v, "device kernel")
+
+    def selftest_bounded_wait(self, limit_cycles, stream=None):
+        _check(self._lib.nm_selftest_bounded_wait(self._h, int(limit_cycles), _stream(stream)),
+               "nm_selftest_bounded_wait")
 
     def launch_count(self, reset=False) -> int:
         return int(self._lib.nm_ctx_launch_count(self._h, 1 if reset else 0))

@@ -20,6 +20,8 @@
 //                 swizzled K-major layout the MMA reads, PWL reciprocal, scaling, store.
 // For L = 512 the S block fills all 512 tensor-memory columns; O then reuses columns
 // 0..63, which are dead once the first 64 exponentials of every row are in P.
+#include <string.h>
+
 #include "nm_common.cuh"
 
 namespace {
@@ -146,6 +148,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     nm_tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_flag;
+    nm_grid_launch_dependents();   // the next kernel may start its set-up
+    nm_grid_dependency_wait();     // Q, K, V come from the previous kernel
     const int n_pchunks = L / 64;
 
     if (warp == 0) {
@@ -376,7 +380,18 @@ nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
     const int64_t grid = (int64_t)d->B * d->heads * (L / BQ);
     if (grid > 0x7fffffffLL) return NM_ERR_SHAPE;
     NmLaunchScope scope(ctx, NM_KERNEL_ATTENTION_TC, 4.0 * (double)d->B * d->heads * (double)L * L * HD, st);
-    kern<<<(unsigned)grid, 32 + 128 * NH, smem, st>>>(tmQ, tmK, tmV, a);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(32 + 128 * NH);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->pdl ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, tmV, a) != cudaSuccess) return NM_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
 }
 

@@ -202,6 +202,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     nm_tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_flag;
+    // set-up done: the next kernel in the stream may begin its own set-up; nothing produced by the
+    // previous kernel has been touched yet, everything below may depend on it
+    nm_grid_launch_dependents();
+    nm_grid_dependency_wait();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -536,14 +540,20 @@ nm_status launch(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
+    cfg.attrs = attr;
+    cfg.numAttrs = 0;
+    if (ctx->pdl) {
+        attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs++;
+    }
     if constexpr (TWO) {
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        attr[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
+        attr[cfg.numAttrs].val.clusterDim.x = 2;
+        attr[cfg.numAttrs].val.clusterDim.y = 1;
+        attr[cfg.numAttrs].val.clusterDim.z = 1;
+        cfg.numAttrs++;
         // persistent: no more clusters than can be resident at once (cached per kernel and smem size)
         static int max_clusters = 0;
         static size_t max_clusters_smem = 0;

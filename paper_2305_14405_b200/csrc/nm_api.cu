@@ -2,6 +2,7 @@
 // validation, kernel selection, and the encoder-layer sequencing.  All arithmetic
 // of the forward pass happens in the kernels this file launches.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -97,6 +98,10 @@ nm_status nm_ctx_create(nm_ctx** out, int device)
         return NM_ERR_CUDA;
     }
     ctx->encode_tiled = fn;
+    {
+        const char* e = getenv("NM_PDL");   // NM_PDL=0 turns programmatic dependent launch off
+        ctx->pdl = (e && e[0] == '0') ? 0 : 1;
+    }
     ctx->prof = new (std::nothrow) NmProfRecord[NM_PROF_MAX];
     if (!ctx->prof) { cudaFree(ctx->d_tables); cudaFree(ctx->d_status); delete ctx; return NM_ERR_CUDA; }
     *out = ctx;
@@ -340,6 +345,13 @@ nm_status nm_layernorm_pwl(nm_ctx* ctx, const void* x, const float* gamma, const
     if (H % 8 != 0) return NM_ERR_SHAPE;
     if (!nm_aligned16(x) || !nm_aligned16(y) || !nm_aligned16(gamma) || !nm_aligned16(beta)) return NM_ERR_ALIGNMENT;
     return nm_launch_layernorm(ctx, x, gamma, beta, y, rows, H, eps, rsqrt_slot, dtype, (cudaStream_t)stream);
+}
+
+nm_status nm_selftest_bounded_wait(nm_ctx* ctx, int64_t limit_cycles, void* stream)
+{
+    if (!ctx) return NM_ERR_INVALID_ARG;
+    if (limit_cycles < 1 || limit_cycles > 4000000000LL) return NM_ERR_SHAPE;
+    return nm_launch_wait_selftest(ctx, (long long)limit_cycles, (cudaStream_t)stream);
 }
 
 nm_status nm_quantize_i8(nm_ctx* ctx, const void* x, nm_dtype dtype, int64_t count, float inv_scale, int8_t* q,

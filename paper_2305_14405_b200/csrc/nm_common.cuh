@@ -43,6 +43,7 @@ struct nm_ctx {
     int prof_count;            // records in use
     int prof_created;          // event pairs created so far (kept for reuse)
     NmProfRecord* prof;        // NM_PROF_MAX records, host memory
+    int pdl;                   // launch kernels with programmatic stream serialization (prologue overlap)
 };
 
 // Brackets one kernel launch with events when profiling is on; counts the launch always.
@@ -163,8 +164,8 @@ __device__ __forceinline__ bool nm_mbar_try_wait(uint64_t* bar, uint32_t parity)
 // records NM_ERR_TIMEOUT in the global status word, raises the CTA's abort flag
 // and returns false.  The caller then skips its remaining work and falls through
 // to the common teardown (no trap, no endless spin).
-__device__ __forceinline__ bool nm_mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                             int* status)
+__device__ __forceinline__ bool nm_mbar_wait_limit(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                   int* status, long long limit_cycles)
 {
     if (nm_mbar_try_wait(bar, parity)) return true;
     long long t0 = clock64();
@@ -173,13 +174,18 @@ __device__ __forceinline__ bool nm_mbar_wait(uint64_t* bar, uint32_t parity, vol
         if (nm_mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > NM_WAIT_LIMIT_CYCLES) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1;
                 atomicExch(status, (int)NM_ERR_TIMEOUT);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool nm_mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                             int* status)
+{
+    return nm_mbar_wait_limit(bar, parity, abort_flag, status, NM_WAIT_LIMIT_CYCLES);
 }
 
 // The same bounded wait for warps that are NOT on the critical issue path (epilogue and
@@ -275,6 +281,15 @@ __device__ __forceinline__ void nm_prefetch_tmap(const CUtensorMap* tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
+
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
+// attribute may start while its predecessor in the stream is still running; it must not touch
+// memory the predecessor produces before nm_grid_dependency_wait() returns (which waits for the
+// predecessor to complete and flush).  nm_grid_launch_dependents() lets the successor's CTAs be
+// scheduled as soon as resources free up, so that its set-up overlaps this kernel's tail.
+// Both are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void nm_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void nm_grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---- tcgen05 ------------------------------------------------------------------
 
@@ -534,6 +549,7 @@ nm_status nm_launch_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int
                               int32_t* idx_out, cudaStream_t st);
 nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
                               int64_t rows, int32_t H, float eps, int32_t slot, nm_dtype dtype, cudaStream_t st);
+nm_status nm_launch_wait_selftest(nm_ctx* ctx, long long limit_cycles, cudaStream_t st);
 nm_status nm_launch_quantize(nm_ctx* ctx, const void* x, nm_dtype dtype, int64_t count, float inv_scale,
                              int8_t* q, cudaStream_t st);
 nm_status nm_launch_linear_simt(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st);

@@ -1,6 +1,8 @@
 // HBM-bound kernels of the PWL forward pass: element-wise table evaluation,
 // LayerNorm with PWL rsqrt, and int8 quantisation.  One read and one write per
 // element, 128-bit accesses, no staging through shared memory needed.
+#include <string.h>
+
 #include "nm_common.cuh"
 
 namespace {
@@ -88,6 +90,8 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restric
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int nvec = H / N;  // H is a multiple of N
     const float inv_h = tab->inv_h, off = tab->off, nm1 = (float)(tab->n - 1);
+    nm_grid_launch_dependents();   // the next kernel may start its set-up
+    nm_grid_dependency_wait();     // x comes from the previous kernel
     uint4 nxt[ITERS];
     if (warp0 < rows) {
 #pragma unroll
@@ -185,6 +189,26 @@ __global__ void __launch_bounds__(256) quantize_kernel(const T* __restrict__ x, 
     }
 }
 
+// One warp waits on a barrier that nothing ever arrives on: exercises the bounded wait every
+// tensor-core kernel relies on.  The wait gives up after `limit_cycles`, records the timeout in
+// the status word and the kernel returns normally (no trap, the context stays usable).
+__global__ void wait_selftest_kernel(int* status, long long limit_cycles, int* reached_end)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        nm_mbar_init(&bar, 1);
+        nm_fence_barrier_init();
+    }
+    __syncthreads();
+    int ok = 1;
+    if (threadIdx.x == 0) ok = nm_mbar_wait_limit(&bar, 0, &abort_flag, status, limit_cycles) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncthreads();
+    if (threadIdx.x == 0) *reached_end = ok ? 2 : 1;   // 1: gave up and fell through to the common exit
+}
+
 template <typename T>
 nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const void* x, const float* gamma, const float* beta, void* y,
                     int64_t rows, int H, float eps, cudaStream_t st)
@@ -197,8 +221,19 @@ nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const void* x, const float*
     int64_t blocks = (rows + 7) / 8;
     if (blocks > (int64_t)ctx->sm_count * 6) blocks = (int64_t)ctx->sm_count * 6;
  NmLaunchScope scope(ctx, NM_KERNEL_LAYERNORM, 2.0 * (double)rows * H * sizeof(T), st);
-#define NM_LN_CASE(I)                                                                                      \
-    layernorm_kernel<T, I><<<(unsigned)blocks, threads, 0, st>>>(tab, (const T*)x, gamma, beta, (T*)y, rows, H, eps)
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->pdl ? 1 : 0;
+    const T* xt = (const T*)x;
+    T* yt = (T*)y;
+#define NM_LN_CASE(I) cudaLaunchKernelEx(&cfg, layernorm_kernel<T, I>, tab, xt, gamma, beta, yt, rows, H, eps)
     if (iters <= 1) NM_LN_CASE(1);
     else if (iters <= 2) NM_LN_CASE(2);
     else if (iters <= 3) NM_LN_CASE(3);
@@ -251,6 +286,16 @@ nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, co
     case NM_F16: return launch_ln<__half>(ctx, tab, x, gamma, beta, y, rows, H, eps, st);
     default: return NM_ERR_UNSUPPORTED;
     }
+}
+
+nm_status nm_launch_wait_selftest(nm_ctx* ctx, long long limit_cycles, cudaStream_t st)
+{
+    // the second word of the status allocation would be cleaner; the kernel only needs one scratch int,
+    // for which the (unused) padding of table slot NM_NUM_SLOTS-1 serves
+    int* scratch = &ctx->d_tables[NM_NUM_SLOTS - 1].pad[0];
+    NmLaunchScope scope(ctx, NM_KERNEL_PWL_APPLY, 0.0, st);
+    wait_selftest_kernel<<<1, 32, 0, st>>>(ctx->d_status, limit_cycles, scratch);
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
 }
 
 nm_status nm_launch_quantize(nm_ctx* ctx, const void* x, nm_dtype dtype, int64_t count, float inv_scale,

@@ -139,3 +139,19 @@ def test_elastic_tables_evaluate_bit_exact(nm, ctx, func, lo, hi, dLx, dK):
     exact = oracle.exact(FUNCS[func], xx)
     t0, _ = oracle_elastic_table(FUNCS[func], lo, hi, dLx, dK, bias_correct=False)
     assert ((t(xx) - exact) ** 2).mean() < ((t0(xx) - exact) ** 2).mean()
+
+
+def test_bounded_wait_times_out_and_context_survives(nm, ctx):
+    """Failure detection without a GPU fault: a wait that can never be satisfied gives up after its
+    limit, the kernel returns normally, the status word carries NM_ERR_TIMEOUT, and the context keeps
+    working."""
+    assert ctx.poll_status() == 0
+    ctx.selftest_bounded_wait(100_000_000)              # ~50 ms of SM clock
+    assert ctx.poll_status() == 7                       # NM_ERR_TIMEOUT, and the word is cleared by the poll
+    assert ctx.poll_status() == 0
+    load_tables_both(ctx, 64, {"gelu": RANGES["gelu"]})
+    x = torch.linspace(-3, 3, 64, device="cuda")
+    y = torch.empty_like(x)
+    ctx.pwl_apply(nm.SLOT_GELU, x, y)                   # the context is still usable
+    torch.cuda.synchronize()
+    assert torch.isfinite(y).all() and ctx.poll_status() == 0
