@@ -172,7 +172,9 @@ nm_status nm_linear_pwl(nm_ctx* ctx, const nm_linear_desc* desc, void* stream);
  * base[b*stride_b + t*stride_t + g*d + c], so the three may point into one packed
  * [B*L, 3*heads*d] projection.  out: device [B*L, heads*d], leading dimension
  * heads*d.  dtype F32, BF16 or F16 (fp32 arithmetic inside).
- * algo as in nm_linear_desc. */
+ * algo: 0 = pick; 1 = CUDA-core kernel; 2 = tensor-core kernel that streams K and V and computes
+ * Q K^T twice (d = 64, L a multiple of 128); 3 = tensor-core kernel that keeps the whole score block
+ * in tensor memory (d = 64, L in {128, 256, 384, 512}). */
 typedef struct {
     int32_t B, L, heads, d;
     nm_dtype dtype;

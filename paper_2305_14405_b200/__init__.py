@@ -20,6 +20,7 @@ F32, BF16, F16, I8 = 0, 1, 2, 3
 SLOT_NONE, SLOT_GELU, SLOT_EXP, SLOT_RECIP, SLOT_RSQRT, SLOT_RELU, SLOT_USER0 = -1, 0, 1, 2, 3, 4, 5
 FUNC_GELU, FUNC_EXP, FUNC_RECIP, FUNC_RSQRT, FUNC_RELU, FUNC_SQRT, FUNC_IDENTITY = range(7)
 ALGO_AUTO, ALGO_SIMT, ALGO_TC, ALGO_TC_1CTA = 0, 1, 2, 3
+ALGO_ATTN_RESIDENT = 3   # attention only: the kernel that keeps the score block in tensor memory
 STATIC_WS_BYTES = 32 << 20
 
 EXPORTS = [

@@ -101,6 +101,8 @@ nm_status nm_ctx_create(nm_ctx** out, int device)
     {
         const char* e = getenv("NM_PDL");   // NM_PDL=0 turns programmatic dependent launch off
         ctx->pdl = (e && e[0] == '0') ? 0 : 1;
+        e = getenv("NM_ATTN_RESIDENT");     // NM_ATTN_RESIDENT=1: algo 0 picks the resident-score attention kernel
+        ctx->attn_resident = (e && e[0] == '1') ? 1 : 0;
     }
     ctx->prof = new (std::nothrow) NmProfRecord[NM_PROF_MAX];
     if (!ctx->prof) { cudaFree(ctx->d_tables); cudaFree(ctx->d_status); delete ctx; return NM_ERR_CUDA; }
@@ -328,9 +330,20 @@ nm_status nm_attention_pwl(nm_ctx* ctx, const nm_attn_desc* d, void* stream)
     if (d->stride_t < (int64_t)d->heads * d->d || d->stride_b < (int64_t)d->L * d->stride_t) return NM_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (d->algo == 1) return nm_launch_attention_simt(ctx, d, st);
-    const bool tc = nm_attention_tc_supported(d);
-    if (d->algo == 2) return tc ? nm_launch_attention_tc(ctx, d, st) : NM_ERR_UNSUPPORTED;
-    return tc ? nm_launch_attention_tc(ctx, d, st) : nm_launch_attention_simt(ctx, d, st);
+    // tensor-core kernels: the streaming one (two CTAs per SM, any L that is a multiple of 128) is the
+    // default; algo 3 selects the one that keeps the whole score block in tensor memory (L <= 512)
+    if (d->algo == 3) return nm_attention_tc_supported(d) ? nm_launch_attention_tc(ctx, d, st) : NM_ERR_UNSUPPORTED;
+    if (d->algo == 0 && ctx->attn_resident && nm_attention_tc_supported(d)) {
+        const nm_status s = nm_launch_attention_tc(ctx, d, st);
+        if (s != NM_ERR_UNSUPPORTED) return s;
+    }
+    const bool tc = nm_attention_stream_supported(d);
+    if (d->algo == 2) return tc ? nm_launch_attention_stream(ctx, d, st) : NM_ERR_UNSUPPORTED;
+    if (tc) {
+        const nm_status s = nm_launch_attention_stream(ctx, d, st);
+        if (s != NM_ERR_UNSUPPORTED) return s;   // else: an exp table too large for shared memory
+    }
+    return nm_launch_attention_simt(ctx, d, st);
 }
 
 nm_status nm_layernorm_pwl(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,

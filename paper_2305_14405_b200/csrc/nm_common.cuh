@@ -44,6 +44,7 @@ struct nm_ctx {
     int prof_created;          // event pairs created so far (kept for reuse)
     NmProfRecord* prof;        // NM_PROF_MAX records, host memory
     int pdl;                   // launch kernels with programmatic stream serialization (prologue overlap)
+    int attn_resident;         // algo 0 prefers the attention kernel with the score block resident in TMEM
 };
 
 // Brackets one kernel launch with events when profiling is on; counts the launch always.
@@ -192,6 +193,7 @@ __device__ __forceinline__ bool nm_mbar_wait(uint64_t* bar, uint32_t parity, vol
 // softmax warps waiting for the tensor core): between polls the thread sleeps, so that a
 // waiting warp does not take issue slots from the single thread that feeds the tensor core
 // on the same scheduler.
+template <unsigned SLEEP_NS = 40>
 __device__ __forceinline__ bool nm_mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                                      int* status)
 {
@@ -199,7 +201,7 @@ __device__ __forceinline__ bool nm_mbar_wait_relaxed(uint64_t* bar, uint32_t par
     long long t0 = clock64();
     uint32_t spins = 0;
     while (true) {
-        __nanosleep(40);
+        __nanosleep(SLEEP_NS);
         if (nm_mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
@@ -558,6 +560,8 @@ bool nm_linear_tc_supported(const nm_linear_desc* d);
 nm_status nm_launch_attention_simt(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
 nm_status nm_launch_attention_tc(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
 bool nm_attention_tc_supported(const nm_attn_desc* d);
+nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
+bool nm_attention_stream_supported(const nm_attn_desc* d);
 nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int Nb, int H, int W, int Cin, int kh,
                            int kw, int stride, int pad, int Ho, int Wo, int Kpad, cudaStream_t st);
 nm_status nm_launch_pad_rows(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, int rows, int K, int Kpad,

@@ -42,18 +42,18 @@ def test_attention_f32_simt(nm, ctx, B, L, h, d):
     assert_close_f32(got, ref, "attention f32")
 
 
-@pytest.mark.parametrize("algo", ["simt", "tc"])
+@pytest.mark.parametrize("algo", ["simt", "tc", "tc_resident"])
 @pytest.mark.parametrize("B,L,h,d,qk", [(2, 128, 12, 64, 0.6), (1, 512, 3, 64, 0.6), (3, 128, 2, 64, 1.5), (1, 256, 2, 64, 1.0),
-                                        (1, 384, 1, 64, 0.8)])
+                                        (1, 384, 1, 64, 0.8), (1, 1024, 2, 64, 0.7)])
 def test_attention_bf16(nm, ctx, algo, B, L, h, d, qk):
     """Scores of different spread: near-uniform rows (the synthetic BERT workload) and peaked ones
     that reach the clamped end segments of the exp table."""
-    a = nm.ALGO_SIMT if algo == "simt" else nm.ALGO_TC
+    a = {"simt": nm.ALGO_SIMT, "tc": nm.ALGO_TC, "tc_resident": nm.ALGO_ATTN_RESIDENT}[algo]
     try:
         got, ref = run(nm, ctx, "bf16", B, L, h, d, a, seed=L + h, qk_scale=qk)
     except nm.NmError as e:
-        if algo == "tc" and e.code == 5 and L not in (128, 512):
-            pytest.skip("tensor-core attention kernel takes L in {128, 512} only")
+        if algo == "tc_resident" and e.code == 5 and L > 512:
+            pytest.skip("the resident-score kernel takes L up to 512 only")
         raise
     assert_close_bf16(got, ref, "attention bf16 %s" % algo)
 
