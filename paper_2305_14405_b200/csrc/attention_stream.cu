@@ -12,13 +12,17 @@
 // shared memory: two CTAs fit on an SM and one CTA's loads, MMAs and barriers overlap the other's
 // arithmetic.  Any L that is a multiple of 128 is supported.
 //
-//   warp 0      TMA producer: Q once; K and V in 64-key chunks through a 6-stage ring, in exactly
-//               the order the MMA warp consumes them (K0..Kn-1, then K0, K1, V0, K2, V1, ...)
-//   warp 1      tcgen05.mma issuer: S chunk = Q K_c^T (128 x 64) into one of two tensor-memory
-//               buffers; in the second sweep also O += P_c V_c (V as an MN-major operand)
-//   warps 2-9   softmax, two per tensor-memory lane quarter, each owning 32 of a chunk's 64
-//               columns: tcgen05.ld, row maximum (sweep 1); PWL exp, row sum, bf16 P tile in the
-//               swizzled K-major layout (sweep 2); PWL reciprocal, scaling, store.
+// The keys are split between two groups of four softmax warps: group g takes chunks g, g+2, ... of
+// 64 keys and owns a score buffer S_g, a P tile and an accumulator O_g (summed in the epilogue), so
+// the two groups form independent pipelines.
+//
+//   warps 0-1   control warp of group 0 / 1: TMA loads (Q; the group's K chunks through two stages,
+//               its V chunks through one) and the tcgen05.mma for S_g = Q K_c^T and O_g += P_c V_c
+//               (V as an MN-major operand).  It sleeps in a named barrier (bar.sync) that the
+//               group's softmax warps signal with bar.arrive, so hand-offs cost no polling.
+//   warps 2-9   softmax, one per tensor-memory lane quarter and group: tcgen05.ld, row maximum
+//               (sweep 1); PWL exp, row sum, bf16 P tile in the swizzled K-major layout (sweep 2);
+//               PWL reciprocal, scaling, store.
 #include <string.h>
 
 #include "nm_common.cuh"
@@ -29,7 +33,6 @@ constexpr int BQ = 128;    // query rows per CTA
 constexpr int HD = 64;     // head dimension
 constexpr int CK = 64;     // keys per chunk
 constexpr int ROWB = 128;  // bytes per tile row (64 x 16-bit)
-constexpr int NS = 6;      // K/V ring stages
 constexpr int STAGE = CK * ROWB;      // 8 KB
 constexpr int PBUF = BQ * ROWB;       // 16 KB
 constexpr int NTHREADS = 320;
@@ -77,23 +80,24 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 {
     constexpr uint32_t IDESC_QK = nm_idesc(1, AT<T>::fmt, 0, 0, BQ, CK);   // S chunk: 128 x 64
     constexpr uint32_t IDESC_PV = nm_idesc(1, AT<T>::fmt, 0, 1, BQ, HD);   // O: 128 x 64, V MN-major
-    constexpr uint32_t TMEM_COLS = 256;                                     // S0 | S1 | O | unused
+    constexpr uint32_t TMEM_COLS = 256;                                     // S0 | S1 | O0 | O1
     constexpr uint32_t O_COL = 128;
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bar_q, bar_o, bar_drain;
-    __shared__ uint64_t bar_kv_full[NS], bar_kv_empty[NS];
-    __shared__ uint64_t bar_s_full[2], bar_s_empty[2], bar_p_full[2], bar_p_empty[2];
+    __shared__ uint64_t bar_q, bar_drain[2];
+    __shared__ uint64_t bar_k_full[2][2], bar_v_full[2], bar_s_full[2], bar_p_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float s_red[2][BQ];
 
     const int L = a.L;
-    const int n = L / CK;  // chunks
+    const int n = L / CK;      // chunks (even: L is a multiple of 128)
+    const int half = n >> 1;   // chunks per group and sweep
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* q_s = base;                       // 16 KB
-    uint8_t* ring = q_s + BQ * ROWB;           // NS x 8 KB
-    uint8_t* p_s = ring + NS * STAGE;          // 2 x 16 KB
+    uint8_t* k_st = q_s + BQ * ROWB;           // [group][2] x 8 KB
+    uint8_t* v_st = k_st + 4 * STAGE;          // [group] x 8 KB
+    uint8_t* p_s = v_st + 2 * STAGE;           // [group] x 16 KB
     float2* rep = reinterpret_cast<float2*>(p_s + 2 * PBUF);   // (n_exp + 1) x 16 copies
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -108,16 +112,12 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         nm_prefetch_tmap(&tmK);
         nm_prefetch_tmap(&tmV);
         nm_mbar_init(&bar_q, 1);
-        nm_mbar_init(&bar_o, 1);
-        nm_mbar_init(&bar_drain, 1);
-        for (int i = 0; i < NS; ++i) {
-            nm_mbar_init(&bar_kv_full[i], 1);
-            nm_mbar_init(&bar_kv_empty[i], 1);
-        }
         for (int i = 0; i < 2; ++i) {
+            nm_mbar_init(&bar_drain[i], 1);
+            nm_mbar_init(&bar_k_full[i][0], 1);
+            nm_mbar_init(&bar_k_full[i][1], 1);
+            nm_mbar_init(&bar_v_full[i], 1);
             nm_mbar_init(&bar_s_full[i], 1);
-            nm_mbar_init(&bar_s_empty[i], 8);
-            nm_mbar_init(&bar_p_full[i], 8);
             nm_mbar_init(&bar_p_empty[i], 1);
         }
         nm_fence_barrier_init();
@@ -141,204 +141,242 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     nm_grid_launch_dependents();   // the next kernel may start its set-up
     nm_grid_dependency_wait();     // Q, K, V come from the previous kernel
 
-    if (warp == 0) {
-        // ------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            nm_mbar_expect_tx(&bar_q, BQ * ROWB);
-            nm_tma_load_3d(q_s, &tmQ, g * HD, qb * BQ, b, &bar_q);
-            auto push = [&](const CUtensorMap* tm, int chunk) {
-                if (!ok) return;
-                // the ring is deep and this warp shares its scheduler with softmax warps: sleep between polls
-                if (!nm_mbar_wait_relaxed<200>(&bar_kv_empty[stage], phase ^ 1u, abortp, a.status)) { ok = false; return; }
-                nm_mbar_expect_tx(&bar_kv_full[stage], STAGE);
-                nm_tma_load_3d(ring + (size_t)stage * STAGE, tm, g * HD, chunk * CK, b, &bar_kv_full[stage]);
-                if (++stage == NS) { stage = 0; phase ^= 1u; }
-            };
-            for (int c = 0; c < n; ++c) push(&tmK, c);        // sweep 1
-            push(&tmK, 0);                                     // sweep 2
-            for (int c = 0; c < n; ++c) {
-                if (c + 1 < n) push(&tmK, c + 1);
-                push(&tmV, c);
+    if (warp < 2) {
+        // ------------------------------------------------ control warp of group `warp`
+        // Runs with all 32 lanes (barrier tests, counters and descriptors stay warp-uniform); one
+        // elected lane issues the TMA and tcgen05 instructions.  It sleeps in a named barrier until
+        // its group's four softmax warps have arrived there, so signalling costs no polling:
+        //   S-consumed(i): chunk i's scores are in registers -> K stage i & 1 is free (load the chunk
+        //                  after next into it) and S is free (issue Q K^T for the next chunk);
+        //   P-ready(j):    the bf16 P tile of the j-th chunk of sweep 2 is in shared memory -> O += P V.
+        const int gi = warp;
+        const uint32_t bar_sc = 2 + 2 * gi, bar_pr = 3 + 2 * gi;
+        auto chunk_of = [&](int i) { return gi + 2 * (i >= half ? i - half : i); };   // i-th chunk of the group, both sweeps
+        uint8_t* my_k = k_st + (size_t)gi * 2 * STAGE;
+        uint8_t* my_v = v_st + (size_t)gi * STAGE;
+        if (nm_elect_one()) {
+            if (gi == 0) {
+                nm_mbar_expect_tx(&bar_q, BQ * ROWB);
+                nm_tma_load_3d(q_s, &tmQ, g * HD, qb * BQ, b, &bar_q);
             }
-            if (!ok) {
-                long long t0 = clock64();  // bounded pause: copies in flight land before teardown
-                while (clock64() - t0 < 4000000LL) {}
+            for (int s = 0; s < 2; ++s) {
+                nm_mbar_expect_tx(&bar_k_full[gi][s], STAGE);
+                nm_tma_load_3d(my_k + (size_t)s * STAGE, &tmK, g * HD, chunk_of(s) * CK, b, &bar_k_full[gi][s]);
             }
+            nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
+            nm_tma_load_3d(my_v, &tmV, g * HD, gi * CK, b, &bar_v_full[gi]);
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            uint32_t t = 0;   // S chunks issued so far; chunk t uses buffer t & 1 for the (t >> 1)-th time (n is even)
-            bool ok = nm_mbar_wait_relaxed<20>(&bar_q, 0, abortp, a.status);
-            const uint64_t qdesc = nm_smem_desc_sw128(nm_smem_u32(q_s));
-            auto qk = [&](int c) {   // S[c & 1] = Q K_c^T
-                if (!ok) return;
-                const int sb = c & 1;
-                if (!nm_mbar_wait_relaxed<20>(&bar_s_empty[sb], ((t >> 1) & 1u) ^ 1u, abortp, a.status)) { ok = false; return; }
-                if (!nm_mbar_wait_relaxed<20>(&bar_kv_full[stage], phase, abortp, a.status)) { ok = false; return; }
-                nm_tc_fence_after();
-                const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32(ring + (size_t)stage * STAGE));
+        __syncwarp();
+        auto wait = [&](uint64_t* bar, uint32_t parity) {
+            return __all_sync(0xffffffffu, nm_mbar_wait_relaxed<20>(bar, parity, abortp, a.status)) != 0;
+        };
+        bool ok = wait(&bar_q, 0);
+        const uint64_t qdesc = nm_smem_desc_sw128(nm_smem_u32(q_s));
+        auto issue_qk = [&](int i) {   // S_g = Q K^T for the group's i-th chunk (K in stage i & 1)
+            if (!ok) return;
+            if (!wait(&bar_k_full[gi][i & 1], (uint32_t)((i >> 1) & 1))) { ok = false; return; }
+            nm_tc_fence_after();
+            const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32(my_k + (size_t)(i & 1) * STAGE));
+            if (nm_elect_one()) {
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    nm_mma_f16(tmem_base + (uint32_t)(sb * CK), qdesc + 2 * k, kdesc + 2 * k, IDESC_QK, k != 0);
-                nm_tc_commit(&bar_kv_empty[stage]);
-                nm_tc_commit(&bar_s_full[sb]);
-                ++t;
-                if (++stage == NS) { stage = 0; phase ^= 1u; }
-            };
-            for (int c = 0; c < n; ++c) qk(c);   // sweep 1: scores for the row maximum
-            qk(0);                               // sweep 2
-            for (int c = 0; c < n && ok; ++c) {
-                if (c + 1 < n) qk(c + 1);
-                if (!ok) break;
-                const int pb = c & 1;
-                if (!nm_mbar_wait_relaxed<20>(&bar_p_full[pb], (uint32_t)((c >> 1) & 1), abortp, a.status)) { ok = false; break; }
-                if (!nm_mbar_wait_relaxed<20>(&bar_kv_full[stage], phase, abortp, a.status)) { ok = false; break; }
-                nm_tc_fence_after();
-                const uint64_t pdesc = nm_smem_desc_sw128(nm_smem_u32(p_s + (size_t)pb * PBUF));
-                const uint32_t v_addr = nm_smem_u32(ring + (size_t)stage * STAGE);
+                    nm_mma_f16(tmem_base + (uint32_t)(gi * CK), qdesc + 2 * k, kdesc + 2 * k, IDESC_QK, k != 0);
+                nm_tc_commit(&bar_s_full[gi]);
+            }
+            __syncwarp();
+        };
+        issue_qk(0);
+        for (int i = 0; i < n; ++i) {
+            asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed(i)
+            if (i + 1 < n) issue_qk(i + 1);
+            if (ok && i + 2 < n && nm_elect_one()) {
+                nm_mbar_expect_tx(&bar_k_full[gi][i & 1], STAGE);
+                nm_tma_load_3d(my_k + (size_t)(i & 1) * STAGE, &tmK, g * HD, chunk_of(i + 2) * CK, b, &bar_k_full[gi][i & 1]);
+            }
+            __syncwarp();
+            if (i >= half) {
+                const int j = i - half;
+                asm volatile("bar.sync %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");   // P-ready(j)
+                if (ok && !wait(&bar_v_full[gi], (uint32_t)(j & 1))) ok = false;
+                if (ok) {
+                    nm_tc_fence_after();
+                    const uint64_t pdesc = nm_smem_desc_sw128(nm_smem_u32(p_s + (size_t)gi * PBUF));
+                    const uint32_t v_addr = nm_smem_u32(my_v);
+                    if (nm_elect_one()) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
-                    nm_mma_f16(tmem_base + O_COL, pdesc + 2 * k, nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB)),
-                               IDESC_PV, (c | k) != 0);
-                nm_tc_commit(&bar_kv_empty[stage]);
-                nm_tc_commit(&bar_p_empty[pb]);
-                if (++stage == NS) { stage = 0; phase ^= 1u; }
+                        for (int k = 0; k < 4; ++k)   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
+                            nm_mma_f16(tmem_base + O_COL + (uint32_t)(gi * HD), pdesc + 2 * k,
+                                       nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB)), IDESC_PV, (j | k) != 0);
+                        nm_tc_commit(&bar_p_empty[gi]);
+                    }
+                    __syncwarp();
+                }
+                if (ok && j + 1 < half) {   // the V stage is free once this P V has completed (nothing else to do until then)
+                    if (!wait(&bar_p_empty[gi], (uint32_t)(j & 1))) ok = false;
+                    if (ok && nm_elect_one()) {
+                        nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
+                        nm_tma_load_3d(my_v, &tmV, g * HD, chunk_of(i + 1) * CK, b, &bar_v_full[gi]);
+                    }
+                    __syncwarp();
+                }
             }
-            if (ok) nm_tc_commit(&bar_o);
-            else {
-                nm_tc_commit(&bar_drain);
+        }
+        if (!ok) {   // after an abort: let copies land and MMAs retire (bounded) before teardown
+            if (nm_elect_one()) {
+                nm_tc_commit(&bar_drain[gi]);
                 long long t0 = clock64();
-                while (!nm_mbar_try_wait(&bar_drain, 0) && clock64() - t0 < 200000000LL) {}
+                while (!nm_mbar_try_wait(&bar_drain[gi], 0) && clock64() - t0 < 200000000LL) {}
+                while (clock64() - t0 < 4000000LL) {}
             }
+            __syncwarp();
         }
     } else {
         // ------------------------------------------------ softmax warps
+        // Warps 2-5 (group 0) take the even chunks, warps 6-9 (group 1) the odd ones; group g owns S
+        // buffer g, P buffer g and accumulator O_g, so the two groups form two independent pipelines.
+        // A warp never blocks on its group: it signals the control warp with bar.arrive.
         const int q = warp & 3;
-        const int h = (warp - 2) >> 2;
+        const int g2 = (warp - 2) >> 2;
         const int row = q * 32 + lane;
-        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 32);
+        const uint32_t bar_sc = 2 + 2 * g2, bar_pr = 3 + 2 * g2;
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g2 * CK);
         const float inv_h = a.t_exp->inv_h, off = a.t_exp->off, nm1 = (float)(a.n_exp - 1);
         // this lane's copy of the replicated table, with the constant of the index trick folded in:
         // (bits << 7) = 0xA0000000 + s*128 (mod 2^32) for bits = 0x4B400000 + s
         const uint32_t rep_lane = nm_smem_u32(rep) + (uint32_t)(lane & 15) * 8u - 0xA0000000u;
         int ok = 1;
-        uint32_t t = 0;   // S chunks consumed so far; chunk t sits in buffer t & 1, its (t >> 1)-th use (n is even)
-        // waits for the next S chunk, loads this warp's 32 columns, hands the buffer back
-        auto load_s = [&](int sb, uint32_t* r) {
-            const uint32_t par = (t >> 1) & 1u;
-            if (lane == 0 && ok) ok = nm_mbar_wait_relaxed(&bar_s_full[sb], par, abortp, a.status) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (ok) {
-                (void)nm_mbar_try_wait(&bar_s_full[sb], par);
-                nm_tc_fence_after();
-                nm_tmem_ld32_async(t_row + (uint32_t)(sb * CK), r);
-                nm_tmem_ld_wait32(r);
-                nm_tc_fence_before();
-                __syncwarp();
-                if (lane == 0) nm_mbar_arrive(&bar_s_empty[sb]);
-                __syncwarp();
+        // All lanes test the barrier; only when it is not yet complete does lane 0 poll (with sleeps).
+        auto wait_all = [&](uint64_t* bar, uint32_t par) {
+            if (!ok) return;
+            const bool done = nm_mbar_try_wait(bar, par);
+            if (!__all_sync(0xffffffffu, done)) {
+                int w = 1;
+                if (lane == 0) w = nm_mbar_wait_relaxed(bar, par, abortp, a.status) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, w, 0);
+                if (ok) (void)nm_mbar_try_wait(bar, par);
             }
-            ++t;
         };
         // ---- sweep 1: the final row maximum
         float m = -INFINITY;
 #pragma unroll 1
-        for (int c = 0; c < n; ++c) {
-            uint32_t r[32];
-            load_s(c & 1, r);
+        for (int i = 0; i < half; ++i) {
+            wait_all(&bar_s_full[g2], (uint32_t)(i & 1));
             if (ok) {
-                float m0 = -INFINITY, m1 = -INFINITY;
+                nm_tc_fence_after();
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    m0 = max3f(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                    m1 = max3f(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t r[32];
+                    nm_tmem_ld32_async(t_row + (uint32_t)(hh * 32), r);
+                    nm_tmem_ld_wait32(r);
+                    if (hh == 1) {   // both halves are in registers: the control warp may overwrite S
+                        nm_tc_fence_before();
+                        asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
+                    }
+                    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+                    for (int k = 0; k < 32; k += 4) {
+                        m0 = max3f(m0, __uint_as_float(r[k]), __uint_as_float(r[k + 1]));
+                        m1 = max3f(m1, __uint_as_float(r[k + 2]), __uint_as_float(r[k + 3]));
+                    }
+                    m = max3f(m, m0, m1);
                 }
-                m = max3f(m, m0, m1);
+            } else {
+                asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
             }
         }
-        s_red[h][row] = m;
+        s_red[g2][row] = m;
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
         m = fmaxf(s_red[0][row], s_red[1][row]);
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
         const float neg_ms = -(m * a.scale);
         float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(g2 * PBUF + row * ROWB);
         // ---- sweep 2: e = PWL_exp(s - m), row sum, P tiles
 #pragma unroll 1
-        for (int c = 0; c < n; ++c) {
-            uint32_t r[32];
-            load_s(c & 1, r);
-            const int pb = c & 1;
-            if (c >= 2 && ok) {
-                const uint32_t par = (uint32_t)(((c >> 1) - 1) & 1);
-                if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_p_empty[pb], par, abortp, a.status) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (ok) (void)nm_mbar_try_wait(&bar_p_empty[pb], par);
-            }
-            if (ok) {
-                const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(pb * PBUF + row * ROWB);
+        for (int j = 0; j < half; ++j) {
+            wait_all(&bar_s_full[g2], (uint32_t)((half + j) & 1));
+            if (ok) nm_tc_fence_after();
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {   // 8 keys = one 16-byte chunk of the P row
-                    float e[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float x = __fmaf_rn(__uint_as_float(r[j * 8 + i]), a.scale, neg_ms);
-                        float u = fmaxf(__fmaf_rn(x, inv_h, off), 0.0f);
-                        if (CLAMP_HI) u = fminf(u, nm1);
-                        // floor(u) sits in the low mantissa bits after a round-down add of 1.5 * 2^23
-                        const uint32_t bits = __float_as_uint(__fadd_rd(u, 12582912.0f));
-                        float kk, bb;
-                        asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(kk), "=f"(bb) : "r"((bits << 7) + rep_lane));
-                        e[i] = __fmaf_rn(kk, x, bb);
-                    }
-                    sum0 += e[0] + e[4];
-                    sum1 += e[1] + e[5];
-                    sum2 += e[2] + e[6];
-                    sum3 += e[3] + e[7];
-                    // chunk index is XORed with the row (128-byte swizzle of the K-major P tile)
-                    const uint32_t addr = prow + (uint32_t)(((h * 4 + j) ^ (row & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(AT<T>::pack(e[0], e[1])),
-                                 "r"(AT<T>::pack(e[2], e[3])), "r"(AT<T>::pack(e[4], e[5])), "r"(AT<T>::pack(e[6], e[7]))
-                                 : "memory");
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t r[32];
+                if (ok) {
+                    nm_tmem_ld32_async(t_row + (uint32_t)(hh * 32), r);
+                    nm_tmem_ld_wait32(r);
                 }
-                nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
-                nm_tc_fence_before();
-                __syncwarp();
-                if (lane == 0) nm_mbar_arrive(&bar_p_full[pb]);
-                __syncwarp();
+                if (hh == 1) {
+                    nm_tc_fence_before();
+                    asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
+                }
+                uint32_t pk[16];   // the half's 32 exponentials, packed to 16 bits
+                if (ok) {
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {   // 8 keys = one 16-byte chunk of the P row
+                        float e[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const float x = __fmaf_rn(__uint_as_float(r[jj * 8 + k]), a.scale, neg_ms);
+                            float u = fmaxf(__fmaf_rn(x, inv_h, off), 0.0f);
+                            if (CLAMP_HI) u = fminf(u, nm1);
+                            // floor(u) sits in the low mantissa bits after a round-down add of 1.5 * 2^23
+                            const uint32_t bits = __float_as_uint(__fadd_rd(u, 12582912.0f));
+                            float kk, bb;
+                            asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(kk), "=f"(bb) : "r"((bits << 7) + rep_lane));
+                            e[k] = __fmaf_rn(kk, x, bb);
+                        }
+                        sum0 += e[0] + e[4];
+                        sum1 += e[1] + e[5];
+                        sum2 += e[2] + e[6];
+                        sum3 += e[3] + e[7];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) pk[jj * 4 + k] = AT<T>::pack(e[2 * k], e[2 * k + 1]);
+                    }
+                }
+                // The stores wait until P V of the group's previous chunk has read the tile; that MMA was
+                // issued just before this chunk began, so the first half's arithmetic runs ahead of it.
+                if (hh == 0 && j >= 1) {
+                    wait_all(&bar_p_empty[g2], (uint32_t)((j - 1) & 1));
+                }
+                if (ok) {
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        // chunk index is XORed with the row (128-byte swizzle of the K-major P tile)
+                        const uint32_t addr = prow + (uint32_t)(((hh * 4 + jj) ^ (row & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pk[jj * 4]), "r"(pk[jj * 4 + 1]),
+                                     "r"(pk[jj * 4 + 2]), "r"(pk[jj * 4 + 3])
+                                     : "memory");
+                    }
+                }
             }
+            nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
+            asm volatile("bar.arrive %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");
         }
-        s_red[h][row] = (sum0 + sum1) + (sum2 + sum3);
+        s_red[g2][row] = (sum0 + sum1) + (sum2 + sum3);
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
         const float sum = s_red[0][row] + s_red[1][row];
+        // ---- r = PWL_recip(sigma), then (O_0 + O_1) * r; each group stores 32 of the 64 channels
+        const int sr = nm_pwl_index(sum, a.t_rcp->inv_h, a.t_rcp->off, (float)(a.t_rcp->n - 1));
+        const float2 kbr = a.t_rcp->kb[sr];
+        const float rinv = __fmaf_rn(kbr.x, sum, kbr.y);
+        wait_all(&bar_p_empty[0], (uint32_t)((half - 1) & 1));   // the last P V of either group has completed
+        wait_all(&bar_p_empty[1], (uint32_t)((half - 1) & 1));
         if (ok) {
-            // ---- r = PWL_recip(sigma), then O * r; each half stores 32 of the 64 channels
-            const int sr = nm_pwl_index(sum, a.t_rcp->inv_h, a.t_rcp->off, (float)(a.t_rcp->n - 1));
-            const float2 kbr = a.t_rcp->kb[sr];
-            const float rinv = __fmaf_rn(kbr.x, sum, kbr.y);
-            if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_o, 0, abortp, a.status) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (ok) {
-                (void)nm_mbar_try_wait(&bar_o, 0);
-                nm_tc_fence_after();
-                T* orow = reinterpret_cast<T*>(a.out) + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
-                          (size_t)g * HD + h * 32;
-                uint32_t r[32];
-                nm_tmem_ld32_async(tmem_base + ((uint32_t)(q * 32) << 16) + O_COL + (uint32_t)(h * 32), r);
-                nm_tmem_ld_wait32(r);
+            nm_tc_fence_after();
+            T* orow = reinterpret_cast<T*>(a.out) + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
+                      (size_t)g * HD + g2 * 32;
+            const uint32_t o_addr = tmem_base + ((uint32_t)(q * 32) << 16) + O_COL + (uint32_t)(g2 * 32);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    uint32_t w[4];
+            for (int jj = 0; jj < 2; ++jj) {   // 16 channels at a time: O_0 and O_1 parts
+                uint32_t r0[16], r1[16];
+                nm_tmem_ld16(o_addr + (uint32_t)(jj * 16), r0);
+                nm_tmem_ld16(o_addr + (uint32_t)(HD + jj * 16), r1);
+                nm_tmem_ld_wait();
+                uint32_t w[8];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        w[i] = AT<T>::pack(__uint_as_float(r[j * 8 + 2 * i]) * rinv, __uint_as_float(r[j * 8 + 2 * i + 1]) * rinv);
-                    reinterpret_cast<uint4*>(orow)[j] = make_uint4(w[0], w[1], w[2], w[3]);
-                }
+                for (int k = 0; k < 8; ++k)
+                    w[k] = AT<T>::pack((__uint_as_float(r0[2 * k]) + __uint_as_float(r1[2 * k])) * rinv,
+                                       (__uint_as_float(r0[2 * k + 1]) + __uint_as_float(r1[2 * k + 1])) * rinv);
+                reinterpret_cast<uint4*>(orow)[2 * jj] = make_uint4(w[0], w[1], w[2], w[3]);
+                reinterpret_cast<uint4*>(orow)[2 * jj + 1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
         }
     }
@@ -381,7 +419,7 @@ nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
     a.out = d->out;
     a.status = ctx->d_status;
     a.n_exp = ctx->h_tables[d->exp_slot].n;
-    const size_t smem = (size_t)BQ * ROWB + (size_t)NS * STAGE + 2 * (size_t)PBUF + (size_t)(a.n_exp + 1) * 16 * sizeof(float2) + 1024;
+    const size_t smem = (size_t)BQ * ROWB + 6 * (size_t)STAGE + 2 * (size_t)PBUF + (size_t)(a.n_exp + 1) * 16 * sizeof(float2) + 1024;
     if (smem > 227 * 1024 - 2048) return NM_ERR_UNSUPPORTED;   // an exp table too large to replicate
     CUtensorMap tmQ, tmK, tmV;
     nm_status s;
