@@ -209,7 +209,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // All 32 lanes run the loop, so that stage, coordinates and addresses stay warp-uniform (the
+        // compiler keeps them in uniform registers); one elected lane issues the copies.
+        {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -217,19 +219,22 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int m0 = (tile / a.num_n_tiles) * TILE_M + (int)rank * BM;
                 const int n0 = (tile % a.num_n_tiles) * BN + (int)rank * B_ROWS;
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
-                    if (!nm_mbar_wait(&bar_empty[stage], phase ^ 1u, abortp, a.status)) { ok = false; break; }
+                    if (!__all_sync(0xffffffffu, nm_mbar_wait(&bar_empty[stage], phase ^ 1u, abortp, a.status))) { ok = false; break; }
                     uint8_t* sa = tiles + (size_t)stage * STAGE_BYTES;
-                    if constexpr (TWO) {
-                        // both CTAs' copies are counted on the leader's barrier
-                        const uint32_t full = nm_mapa(nm_smem_u32(&bar_full[stage]), 0);
-                        if (rank == 0) nm_mbar_expect_tx(&bar_full[stage], 2 * STAGE_BYTES);
-                        nm_tma_load_2d_2cta(sa, &tmA, kb * BK_ELEMS, m0, full);
-                        nm_tma_load_2d_2cta(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, full);
-                    } else {
-                        nm_mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
-                        nm_tma_load_2d(sa, &tmA, kb * BK_ELEMS, m0, &bar_full[stage]);
-                        nm_tma_load_2d(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, &bar_full[stage]);
+                    if (nm_elect_one()) {
+                        if constexpr (TWO) {
+                            // both CTAs' copies are counted on the leader's barrier
+                            const uint32_t full = nm_mapa(nm_smem_u32(&bar_full[stage]), 0);
+                            if (rank == 0) nm_mbar_expect_tx(&bar_full[stage], 2 * STAGE_BYTES);
+                            nm_tma_load_2d_2cta(sa, &tmA, kb * BK_ELEMS, m0, full);
+                            nm_tma_load_2d_2cta(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, full);
+                        } else {
+                            nm_mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
+                            nm_tma_load_2d(sa, &tmA, kb * BK_ELEMS, m0, &bar_full[stage]);
+                            nm_tma_load_2d(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, &bar_full[stage]);
+                        }
                     }
+                    __syncwarp();
                     if (++stage == stages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -240,50 +245,61 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (the leader CTA of a pair)
-        if (lane == 0 && rank == 0) {
+        // All 32 lanes run the loop (waits, counters and descriptors stay warp-uniform); one elected
+        // lane, always the same, issues the tcgen05 instructions and their commits.
+        if (rank == 0) {
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
             for (int tile = tile_first; ok && tile < a.num_tiles; tile += tile_step) {
-                if (!(TWO ? nm_mbar_wait_cluster(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status)
-                          : nm_mbar_wait(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, TWO ? nm_mbar_wait_cluster(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status)
+                                                 : nm_mbar_wait(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status))) { ok = false; break; }
                 nm_tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
-                    if (!nm_mbar_wait(&bar_full[stage], phase, abortp, a.status)) { ok = false; break; }
+                    if (!__all_sync(0xffffffffu, nm_mbar_wait(&bar_full[stage], phase, abortp, a.status))) { ok = false; break; }
                     nm_tc_fence_after();
                     const uint32_t sa = nm_smem_u32(tiles + (size_t)stage * STAGE_BYTES);
                     const uint64_t adesc = nm_smem_desc_sw128(sa);
                     const uint64_t bdesc = nm_smem_desc_sw128(sa + A_BYTES);
+                    if (nm_elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {  // 4 x 32 bytes of K per 128-byte row
-                        const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-                        if constexpr (TWO) {
-                            if constexpr (TcIn<InT>::is_int) nm_mma_i8_2cta(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
-                            else nm_mma_f16_2cta(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
-                        } else {
-                            if constexpr (TcIn<InT>::is_int) nm_mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
-                            else nm_mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                        for (int k = 0; k < 4; ++k) {  // 4 x 32 bytes of K per 128-byte row
+                            const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
+                            if constexpr (TWO) {
+                                if constexpr (TcIn<InT>::is_int) nm_mma_i8_2cta(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                                else nm_mma_f16_2cta(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                            } else {
+                                if constexpr (TcIn<InT>::is_int) nm_mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                                else nm_mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, accum);
+                            }
                         }
+                        // smem stage reusable (in both CTAs of a pair) once these MMAs retire
+                        if constexpr (TWO) nm_tc_commit2(&bar_empty[stage], 3);
+                        else nm_tc_commit(&bar_empty[stage]);
                     }
-                    // smem stage reusable (in both CTAs of a pair) once these MMAs retire
-                    if constexpr (TWO) nm_tc_commit2(&bar_empty[stage], 3);
-                    else nm_tc_commit(&bar_empty[stage]);
+                    __syncwarp();
                     if (++stage == stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                if constexpr (TWO) nm_tc_commit2(&bar_acc_full[buf], 3);
-                else nm_tc_commit(&bar_acc_full[buf]);
+                if (nm_elect_one()) {
+                    if constexpr (TWO) nm_tc_commit2(&bar_acc_full[buf], 3);
+                    else nm_tc_commit(&bar_acc_full[buf]);
+                }
+                __syncwarp();
                 buf ^= 1;
                 if (buf == 0) acc_phase ^= 1u;
             }
             if (!ok) {
-                if constexpr (TWO) nm_tc_commit2(&bar_drain, 1);
-                else nm_tc_commit(&bar_drain);
-                long long t0 = clock64();
-                while (!nm_mbar_try_wait(&bar_drain, 0) && clock64() - t0 < 200000000LL) {}
+                if (nm_elect_one()) {
+                    if constexpr (TWO) nm_tc_commit2(&bar_drain, 1);
+                    else nm_tc_commit(&bar_drain);
+                    long long t0 = clock64();
+                    while (!nm_mbar_try_wait(&bar_drain, 0) && clock64() - t0 < 200000000LL) {}
+                }
+                __syncwarp();
             }
         }
     } else {
