@@ -162,6 +162,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint8_t* stage_out = tiles + (size_t)stages * STAGE_BYTES;   // 8 x 4 KB
     uint8_t* stage_res = stage_out + NUM_EPI_WARPS * STAGE_BUF;   // 8 x 4 KB when a residual is given
     float2* rep = reinterpret_cast<float2*>(stage_res + (a.has_res ? NUM_EPI_WARPS * STAGE_BUF : 0));
+    // per epilogue warp: bias (128 floats) and, for int8, a_scale * w_scale (128 floats) of its tile columns
+    float* vec_s = reinterpret_cast<float*>(rep + (size_t)a.n_seg * 32);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = TWO ? nm_cluster_ctarank() : 0u;  // 0 = leader of the pair
@@ -328,13 +330,48 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             nm_tma_load_2d(my_res, &tmR, n0, m0 + q * 32, &bar_res[e]);
         }
         int ok = 1;
+        // All lanes test a barrier; only when it is not yet complete does lane 0 poll (with sleeps).
+        auto wait_all = [&](uint64_t* bar, uint32_t par) {
+            const bool done = nm_mbar_try_wait(bar, par);
+            if (!__all_sync(0xffffffffu, done)) {
+                int w = 1;
+                if (lane == 0) w = nm_mbar_wait_relaxed(bar, par, abortp, a.status) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, w, 0);
+                if (ok) (void)nm_mbar_try_wait(bar, par);  // every lane observes the phase itself
+            }
+        };
+        // Per-column vectors of the warp's 128 tile columns go through shared memory: lane l fetches
+        // columns 4l..4l+3 one tile ahead (the latency hides behind the current tile), and the chunk
+        // loop reads them as broadcasts.
+        const bool use_vec = a.bias != nullptr || TcIn<InT>::is_int;
+        float* my_vec = vec_s + e * 256;
+        float4 nxt_b = make_float4(0.f, 0.f, 0.f, 0.f), nxt_s = make_float4(0.f, 0.f, 0.f, 0.f);
+        auto fetch_vec = [&](int t) {
+            nxt_b = make_float4(0.f, 0.f, 0.f, 0.f);
+            nxt_s = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (!use_vec || t >= a.num_tiles) return;
+            const int64_t col = (int64_t)(t % a.num_n_tiles) * BN + half * (BN / 2) + 4 * lane;
+            if (col < a.N) {
+                if (a.bias) nxt_b = __ldg(reinterpret_cast<const float4*>(a.bias + col));
+                if constexpr (TcIn<InT>::is_int) {
+                    const float4 ws = __ldg(reinterpret_cast<const float4*>(a.w_scale + col));
+                    nxt_s = make_float4(a.a_scale * ws.x, a.a_scale * ws.y, a.a_scale * ws.z, a.a_scale * ws.w);
+                }
+            }
+        };
+        fetch_vec(tile_first);
         for (int tile = tile_first; ok && tile < a.num_tiles; tile += tile_step) {
             const int m0 = (tile / a.num_n_tiles) * TILE_M + (int)rank * BM;
             const int n0 = (tile % a.num_n_tiles) * BN + half * (BN / 2);
-            if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_acc_full[buf], acc_phase, abortp, a.status) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (use_vec) {
+                __syncwarp();   // the previous tile's reads of my_vec are done
+                *reinterpret_cast<float4*>(my_vec + 4 * lane) = nxt_b;
+                if constexpr (TcIn<InT>::is_int) *reinterpret_cast<float4*>(my_vec + 128 + 4 * lane) = nxt_s;
+                __syncwarp();
+                fetch_vec(tile + tile_step);
+            }
+            wait_all(&bar_acc_full[buf], acc_phase);
             if (!ok) break;
-            (void)nm_mbar_try_wait(&bar_acc_full[buf], acc_phase);  // every lane observes the phase itself
             nm_tc_fence_after();
             const int64_t row = (int64_t)m0 + q * 32 + lane;
             const bool row_ok = row < a.M;
@@ -346,9 +383,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 uint32_t packed[32];
                 uint32_t rsv[32];
                 if (has_res) {
-                    if (lane == 0) ok = nm_mbar_wait_relaxed(&bar_res[e], res_phase, abortp, a.status) ? 1 : 0;
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (ok) (void)nm_mbar_try_wait(&bar_res[e], res_phase);  // every lane observes the phase itself
+                    wait_all(&bar_res[e], res_phase);
                     res_phase ^= 1u;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
@@ -399,29 +434,25 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if constexpr (TcIn<InT>::is_int) {
 #pragma unroll
                         for (int i = 0; i < 32; i += 4) {
-                            float4 ws = make_float4(0.f, 0.f, 0.f, 0.f), bs = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (col0 + i < a.N) {
-                                ws = __ldg(reinterpret_cast<const float4*>(a.w_scale + col0 + i));
-                                if (a.bias) bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
-                                if (a.acc_dump && row_ok)
-                                    *reinterpret_cast<int4*>(a.acc_dump + row * a.N + col0 + i) =
-                                        make_int4((int)r[cur][i], (int)r[cur][i + 1], (int)r[cur][i + 2], (int)r[cur][i + 3]);
-                            }
-                            v[i] = __fmaf_rn((float)(int)r[cur][i], a.a_scale * ws.x, bs.x);
-                            v[i + 1] = __fmaf_rn((float)(int)r[cur][i + 1], a.a_scale * ws.y, bs.y);
-                            v[i + 2] = __fmaf_rn((float)(int)r[cur][i + 2], a.a_scale * ws.z, bs.z);
-                            v[i + 3] = __fmaf_rn((float)(int)r[cur][i + 3], a.a_scale * ws.w, bs.w);
+                            // a_scale * w_scale and bias of columns beyond N are zero
+                            const float4 ws = *reinterpret_cast<const float4*>(my_vec + 128 + c * 32 + i);
+                            const float4 bs = *reinterpret_cast<const float4*>(my_vec + c * 32 + i);
+                            if (a.acc_dump && row_ok && col0 + i < a.N)
+                                *reinterpret_cast<int4*>(a.acc_dump + row * a.N + col0 + i) =
+                                    make_int4((int)r[cur][i], (int)r[cur][i + 1], (int)r[cur][i + 2], (int)r[cur][i + 3]);
+                            v[i] = __fmaf_rn((float)(int)r[cur][i], ws.x, bs.x);
+                            v[i + 1] = __fmaf_rn((float)(int)r[cur][i + 1], ws.y, bs.y);
+                            v[i + 2] = __fmaf_rn((float)(int)r[cur][i + 2], ws.z, bs.z);
+                            v[i + 3] = __fmaf_rn((float)(int)r[cur][i + 3], ws.w, bs.w);
                         }
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[cur][i]);
                         if (a.bias) {
 #pragma unroll
-                            for (int i = 0; i < 32; i += 4) {
-                                if (col0 + i < a.N) {
-                                    const float4 bs = __ldg(reinterpret_cast<const float4*>(a.bias + col0 + i));
-                                    v[i] += bs.x; v[i + 1] += bs.y; v[i + 2] += bs.z; v[i + 3] += bs.w;
-                                }
+                            for (int i = 0; i < 32; i += 4) {   // zero beyond N
+                                const float4 bs = *reinterpret_cast<const float4*>(my_vec + c * 32 + i);
+                                v[i] += bs.x; v[i + 1] += bs.y; v[i + 2] += bs.z; v[i + 3] += bs.w;
                             }
                         }
                     }
@@ -529,7 +560,8 @@ nm_status launch(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
     a.num_tiles = (int)(m_tiles * a.num_n_tiles);
     a.num_k_blocks = (int)((d->K + bk - 1) / bk);
     const size_t table_bytes = (size_t)a.n_seg * 32 * sizeof(float2);
-    const size_t staging = (size_t)NUM_EPI_WARPS * STAGE_BUF * (a.has_res ? 2 : 1);
+    const size_t vec_bytes = (d->bias || TcIn<InT>::is_int) ? (size_t)NUM_EPI_WARPS * 256 * sizeof(float) : 0;
+    const size_t staging = (size_t)NUM_EPI_WARPS * STAGE_BUF * (a.has_res ? 2 : 1) + vec_bytes;
     const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - table_bytes - staging;
     int stages = (int)(budget / STAGE_BYTES);
     if (stages > MAX_STAGES) stages = MAX_STAGES;

@@ -390,9 +390,12 @@ __device__ __forceinline__ uint32_t nm_mapa(uint32_t addr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
+// Arrival on a barrier that may live in the peer CTA.  Default (CTA-scope) release: what the arrival
+// orders here are tcgen05 operations, which tcgen05.fence::before_thread_sync has already ordered; a
+// cluster-scope release would in addition wait for every earlier global write of the thread.
 __device__ __forceinline__ void nm_mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void nm_cluster_sync()
 {
