@@ -121,6 +121,21 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             nm_mbar_init(&bar_p_empty[i], 1);
         }
         nm_fence_barrier_init();
+        // The first copies go out before the rest of the set-up (tensor-memory allocation, table
+        // replication, block barrier), so that their latency overlaps it: Q, both groups' first two
+        // K chunks (the group's i-th chunk is chunk g + 2i) and first V chunk.
+        nm_grid_dependency_wait();   // Q, K, V come from the previous kernel
+        nm_mbar_expect_tx(&bar_q, BQ * ROWB);
+        nm_tma_load_3d(q_s, &tmQ, g * HD, qb * BQ, b, &bar_q);
+        for (int gi = 0; gi < 2; ++gi) {
+            for (int st = 0; st < 2; ++st) {
+                const int chunk = (st < half) ? gi + 2 * st : gi;   // half == 1: the second is sweep 2's first
+                nm_mbar_expect_tx(&bar_k_full[gi][st], STAGE);
+                nm_tma_load_3d(k_st + (size_t)(gi * 2 + st) * STAGE, &tmK, g * HD, chunk * CK, b, &bar_k_full[gi][st]);
+            }
+            nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
+            nm_tma_load_3d(v_st + (size_t)gi * STAGE, &tmV, g * HD, gi * CK, b, &bar_v_full[gi]);
+        }
     }
     if (warp == 1) {
         nm_tmem_alloc(&tmem_slot, TMEM_COLS);
@@ -154,19 +169,6 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         auto chunk_of = [&](int i) { return gi + 2 * (i >= half ? i - half : i); };   // i-th chunk of the group, both sweeps
         uint8_t* my_k = k_st + (size_t)gi * 2 * STAGE;
         uint8_t* my_v = v_st + (size_t)gi * STAGE;
-        if (nm_elect_one()) {
-            if (gi == 0) {
-                nm_mbar_expect_tx(&bar_q, BQ * ROWB);
-                nm_tma_load_3d(q_s, &tmQ, g * HD, qb * BQ, b, &bar_q);
-            }
-            for (int s = 0; s < 2; ++s) {
-                nm_mbar_expect_tx(&bar_k_full[gi][s], STAGE);
-                nm_tma_load_3d(my_k + (size_t)s * STAGE, &tmK, g * HD, chunk_of(s) * CK, b, &bar_k_full[gi][s]);
-            }
-            nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
-            nm_tma_load_3d(my_v, &tmV, g * HD, gi * CK, b, &bar_v_full[gi]);
-        }
-        __syncwarp();
         auto wait = [&](uint64_t* bar, uint32_t parity) {
             return __all_sync(0xffffffffu, nm_mbar_wait_relaxed<20>(bar, parity, abortp, a.status)) != 0;
         };
