@@ -12,9 +12,11 @@
 // shared memory: two CTAs fit on an SM and one CTA's loads, MMAs and barriers overlap the other's
 // arithmetic.  Any L that is a multiple of 128 is supported.
 //
-// The keys are split between two groups of four softmax warps: group g takes chunks g, g+2, ... of
-// 64 keys and owns a score buffer S_g, a P tile and an accumulator O_g (summed in the epilogue), so
-// the two groups form independent pipelines.
+// The keys are split between two groups of four softmax warps, which form independent pipelines:
+// group g owns 128 tensor-memory columns [S_g | O_g], two K stages, a V stage and a P tile.  In
+// sweep 1 it takes the 128-key chunks g, g+2, ... (scores over all 128 columns, K staged in its two
+// K stages and, alternately, in its P tile); in sweep 2 the 64-key chunks g, g+2, ... (scores in
+// S_g, accumulator O_g; the two accumulators are summed in the epilogue).
 //
 //   warps 0-1   control warp of group 0 / 1: TMA loads (Q; the group's K chunks through two stages,
 //               its V chunks through one) and the tcgen05.mma for S_g = Q K_c^T and O_g += P_c V_c
@@ -80,19 +82,22 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 {
     constexpr uint32_t IDESC_QK = nm_idesc(1, AT<T>::fmt, 0, 0, BQ, CK);   // S chunk: 128 x 64
     constexpr uint32_t IDESC_PV = nm_idesc(1, AT<T>::fmt, 0, 1, BQ, HD);   // O: 128 x 64, V MN-major
-    constexpr uint32_t TMEM_COLS = 256;                                     // S0 | S1 | O0 | O1
-    constexpr uint32_t O_COL = 128;
+    constexpr uint32_t IDESC_QK1 = nm_idesc(1, AT<T>::fmt, 0, 0, BQ, 2 * CK);   // sweep 1: 128 x 128
+    constexpr uint32_t TMEM_COLS = 256;   // S0 | O0 | S1 | O1; sweep 1 writes 128 keys over [S_g | O_g]
+    constexpr uint32_t GRP_COLS = 128;    // tensor-memory columns of a group
+    constexpr uint32_t O_OFF = 64;        // O_g within the group's columns
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_q, bar_drain[2];
-    __shared__ uint64_t bar_k_full[2][2], bar_v_full[2], bar_s_full[2], bar_p_empty[2];
+    __shared__ uint64_t bar_k_full[2][2], bar_k1_full[2][2], bar_v_full[2], bar_s_full[2], bar_p_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float s_red[2][BQ];
 
     const int L = a.L;
     const int n = L / CK;      // chunks (even: L is a multiple of 128)
-    const int half = n >> 1;   // chunks per group and sweep
+    const int half = n >> 1;   // chunks per group in sweep 2
+    const int n128 = L / (2 * CK);   // 128-key chunks of sweep 1: group g takes g, g+2, ...
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* q_s = base;                       // 16 KB
     uint8_t* k_st = q_s + BQ * ROWB;           // [group][2] x 8 KB
@@ -116,22 +121,28 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             nm_mbar_init(&bar_drain[i], 1);
             nm_mbar_init(&bar_k_full[i][0], 1);
             nm_mbar_init(&bar_k_full[i][1], 1);
+            nm_mbar_init(&bar_k1_full[i][0], 1);
+            nm_mbar_init(&bar_k1_full[i][1], 1);
             nm_mbar_init(&bar_v_full[i], 1);
             nm_mbar_init(&bar_s_full[i], 1);
             nm_mbar_init(&bar_p_empty[i], 1);
         }
         nm_fence_barrier_init();
         // The first copies go out before the rest of the set-up (tensor-memory allocation, table
-        // replication, block barrier), so that their latency overlaps it: Q, both groups' first two
-        // K chunks (the group's i-th chunk is chunk g + 2i) and first V chunk.
+        // replication, block barrier), so that their latency overlaps it: Q, each group's first two
+        // 128-key chunks of sweep 1 (stage 0 = the group's two K stages, stage 1 = its P tile, which
+        // sweep 1 does not use otherwise) and its first V chunk.
         nm_grid_dependency_wait();   // Q, K, V come from the previous kernel
         nm_mbar_expect_tx(&bar_q, BQ * ROWB);
         nm_tma_load_3d(q_s, &tmQ, g * HD, qb * BQ, b, &bar_q);
         for (int gi = 0; gi < 2; ++gi) {
             for (int st = 0; st < 2; ++st) {
-                const int chunk = (st < half) ? gi + 2 * st : gi;   // half == 1: the second is sweep 2's first
-                nm_mbar_expect_tx(&bar_k_full[gi][st], STAGE);
-                nm_tma_load_3d(k_st + (size_t)(gi * 2 + st) * STAGE, &tmK, g * HD, chunk * CK, b, &bar_k_full[gi][st]);
+                const int c128 = gi + 2 * st;
+                if (c128 >= n128) break;
+                uint8_t* dst = st == 0 ? k_st + (size_t)gi * 2 * STAGE : p_s + (size_t)gi * PBUF;
+                nm_mbar_expect_tx(&bar_k1_full[gi][st], 2 * STAGE);
+                nm_tma_load_3d(dst, &tmK, g * HD, c128 * 2 * CK, b, &bar_k1_full[gi][st]);
+                nm_tma_load_3d(dst + STAGE, &tmK, g * HD, c128 * 2 * CK + CK, b, &bar_k1_full[gi][st]);
             }
             nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
             nm_tma_load_3d(v_st + (size_t)gi * STAGE, &tmV, g * HD, gi * CK, b, &bar_v_full[gi]);
@@ -166,61 +177,92 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         //   P-ready(j):    the bf16 P tile of the j-th chunk of sweep 2 is in shared memory -> O += P V.
         const int gi = warp;
         const uint32_t bar_sc = 2 + 2 * gi, bar_pr = 3 + 2 * gi;
-        auto chunk_of = [&](int i) { return gi + 2 * (i >= half ? i - half : i); };   // i-th chunk of the group, both sweeps
+        const int cnt1 = (n128 - gi + 1) >> 1;   // the group's 128-key chunks in sweep 1
         uint8_t* my_k = k_st + (size_t)gi * 2 * STAGE;
         uint8_t* my_v = v_st + (size_t)gi * STAGE;
+        uint8_t* my_p = p_s + (size_t)gi * PBUF;
+        const uint32_t my_tmem = tmem_base + (uint32_t)gi * GRP_COLS;
         auto wait = [&](uint64_t* bar, uint32_t parity) {
             return __all_sync(0xffffffffu, nm_mbar_wait_relaxed<20>(bar, parity, abortp, a.status)) != 0;
         };
         bool ok = wait(&bar_q, 0);
         const uint64_t qdesc = nm_smem_desc_sw128(nm_smem_u32(q_s));
-        auto issue_qk = [&](int i) {   // S_g = Q K^T for the group's i-th chunk (K in stage i & 1)
+        // ---- sweep 1: [S_g | O_g] = Q K^T for 128 keys at a time; K stage i & 1 (0: the two K stages
+        // taken together, 1: the P tile)
+        auto issue_qk1 = [&](int i) {
             if (!ok) return;
-            if (!wait(&bar_k_full[gi][i & 1], (uint32_t)((i >> 1) & 1))) { ok = false; return; }
+            if (!wait(&bar_k1_full[gi][i & 1], (uint32_t)((i >> 1) & 1))) { ok = false; return; }
             nm_tc_fence_after();
-            const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32(my_k + (size_t)(i & 1) * STAGE));
+            const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32((i & 1) ? my_p : my_k));
             if (nm_elect_one()) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    nm_mma_f16(tmem_base + (uint32_t)(gi * CK), qdesc + 2 * k, kdesc + 2 * k, IDESC_QK, k != 0);
+                for (int k = 0; k < 4; ++k) nm_mma_f16(my_tmem, qdesc + 2 * k, kdesc + 2 * k, IDESC_QK1, k != 0);
                 nm_tc_commit(&bar_s_full[gi]);
             }
             __syncwarp();
         };
-        issue_qk(0);
-        for (int i = 0; i < n; ++i) {
-            asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed(i)
-            if (i + 1 < n) issue_qk(i + 1);
-            if (ok && i + 2 < n && nm_elect_one()) {
-                nm_mbar_expect_tx(&bar_k_full[gi][i & 1], STAGE);
-                nm_tma_load_3d(my_k + (size_t)(i & 1) * STAGE, &tmK, g * HD, chunk_of(i + 2) * CK, b, &bar_k_full[gi][i & 1]);
+        if (cnt1 > 0) issue_qk1(0);
+        for (int i = 0; i < cnt1; ++i) {
+            asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed: chunk i is in registers
+            if (i + 1 < cnt1) issue_qk1(i + 1);
+            if (ok && i + 2 < cnt1 && nm_elect_one()) {   // its MMAs are complete: the stage takes the chunk after next
+                uint8_t* dst = (i & 1) ? my_p : my_k;
+                const int key0 = (gi + 2 * (i + 2)) * 2 * CK;
+                nm_mbar_expect_tx(&bar_k1_full[gi][i & 1], 2 * STAGE);
+                nm_tma_load_3d(dst, &tmK, g * HD, key0, b, &bar_k1_full[gi][i & 1]);
+                nm_tma_load_3d(dst + STAGE, &tmK, g * HD, key0 + CK, b, &bar_k1_full[gi][i & 1]);
             }
             __syncwarp();
-            if (i >= half) {
-                const int j = i - half;
-                asm volatile("bar.sync %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");   // P-ready(j)
-                if (ok && !wait(&bar_v_full[gi], (uint32_t)(j & 1))) ok = false;
-                if (ok) {
-                    nm_tc_fence_after();
-                    const uint64_t pdesc = nm_smem_desc_sw128(nm_smem_u32(p_s + (size_t)gi * PBUF));
-                    const uint32_t v_addr = nm_smem_u32(my_v);
-                    if (nm_elect_one()) {
+        }
+        // ---- sweep 2: the group's j-th chunk is the 64 keys of chunk g + 2j; K stage j & 1
+        auto load_k = [&](int j) {
+            if (ok && nm_elect_one()) {
+                nm_mbar_expect_tx(&bar_k_full[gi][j & 1], STAGE);
+                nm_tma_load_3d(my_k + (size_t)(j & 1) * STAGE, &tmK, g * HD, (gi + 2 * j) * CK, b, &bar_k_full[gi][j & 1]);
+            }
+            __syncwarp();
+        };
+        auto issue_qk = [&](int j) {   // S_g = Q K^T
+            if (!ok) return;
+            if (!wait(&bar_k_full[gi][j & 1], (uint32_t)((j >> 1) & 1))) { ok = false; return; }
+            nm_tc_fence_after();
+            const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32(my_k + (size_t)(j & 1) * STAGE));
+            if (nm_elect_one()) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
-                            nm_mma_f16(tmem_base + O_COL + (uint32_t)(gi * HD), pdesc + 2 * k,
-                                       nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB)), IDESC_PV, (j | k) != 0);
-                        nm_tc_commit(&bar_p_empty[gi]);
-                    }
-                    __syncwarp();
+                for (int k = 0; k < 4; ++k) nm_mma_f16(my_tmem, qdesc + 2 * k, kdesc + 2 * k, IDESC_QK, k != 0);
+                nm_tc_commit(&bar_s_full[gi]);
+            }
+            __syncwarp();
+        };
+        load_k(0);   // every MMA of sweep 1 has completed: the K stages are free
+        if (half > 1) load_k(1);
+        issue_qk(0);
+        for (int j = 0; j < half; ++j) {
+            asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed(j)
+            if (j + 1 < half) issue_qk(j + 1);
+            if (j + 2 < half) load_k(j + 2);
+            asm volatile("bar.sync %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");   // P-ready(j)
+            if (ok && !wait(&bar_v_full[gi], (uint32_t)(j & 1))) ok = false;
+            if (ok) {
+                nm_tc_fence_after();
+                const uint64_t pdesc = nm_smem_desc_sw128(nm_smem_u32(my_p));
+                const uint32_t v_addr = nm_smem_u32(my_v);
+                if (nm_elect_one()) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
+                        nm_mma_f16(my_tmem + O_OFF, pdesc + 2 * k, nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB)),
+                                   IDESC_PV, (j | k) != 0);
+                    nm_tc_commit(&bar_p_empty[gi]);
                 }
-                if (ok && j + 1 < half) {   // the V stage is free once this P V has completed (nothing else to do until then)
-                    if (!wait(&bar_p_empty[gi], (uint32_t)(j & 1))) ok = false;
-                    if (ok && nm_elect_one()) {
-                        nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
-                        nm_tma_load_3d(my_v, &tmV, g * HD, chunk_of(i + 1) * CK, b, &bar_v_full[gi]);
-                    }
-                    __syncwarp();
+                __syncwarp();
+            }
+            if (ok && j + 1 < half) {   // the V stage is free once this P V has completed (nothing else to do until then)
+                if (!wait(&bar_p_empty[gi], (uint32_t)(j & 1))) ok = false;
+                if (ok && nm_elect_one()) {
+                    nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
+                    nm_tma_load_3d(my_v, &tmV, g * HD, (gi + 2 * (j + 1)) * CK, b, &bar_v_full[gi]);
                 }
+                __syncwarp();
             }
         }
         if (!ok) {   // after an abort: let copies land and MMAs retire (bounded) before teardown
@@ -241,7 +283,8 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         const int g2 = (warp - 2) >> 2;
         const int row = q * 32 + lane;
         const uint32_t bar_sc = 2 + 2 * g2, bar_pr = 3 + 2 * g2;
-        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g2 * CK);
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g2 * GRP_COLS;
+        const int cnt1 = (n128 - g2 + 1) >> 1;   // the group's 128-key chunks in sweep 1
         const float inv_h = a.t_exp->inv_h, off = a.t_exp->off, nm1 = (float)(a.n_exp - 1);
         // this lane's copy of the replicated table, with the constant of the index trick folded in:
         // (bits << 7) = 0xA0000000 + s*128 (mod 2^32) for bits = 0x4B400000 + s
@@ -261,16 +304,16 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         // ---- sweep 1: the final row maximum
         float m = -INFINITY;
 #pragma unroll 1
-        for (int i = 0; i < half; ++i) {
+        for (int i = 0; i < cnt1; ++i) {
             wait_all(&bar_s_full[g2], (uint32_t)(i & 1));
             if (ok) {
                 nm_tc_fence_after();
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
+                for (int hh = 0; hh < 4; ++hh) {   // 128 keys: the scores span [S_g | O_g]
                     uint32_t r[32];
                     nm_tmem_ld32_async(t_row + (uint32_t)(hh * 32), r);
                     nm_tmem_ld_wait32(r);
-                    if (hh == 1) {   // both halves are in registers: the control warp may overwrite S
+                    if (hh == 3) {   // all of it is in registers: the control warp may overwrite S
                         nm_tc_fence_before();
                         asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
                     }
@@ -296,7 +339,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         // ---- sweep 2: e = PWL_exp(s - m), row sum, P tiles
 #pragma unroll 1
         for (int j = 0; j < half; ++j) {
-            wait_all(&bar_s_full[g2], (uint32_t)((half + j) & 1));
+            wait_all(&bar_s_full[g2], (uint32_t)((cnt1 + j) & 1));
             if (ok) nm_tc_fence_after();
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
@@ -365,12 +408,12 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             nm_tc_fence_after();
             T* orow = reinterpret_cast<T*>(a.out) + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
                       (size_t)g * HD + g2 * 32;
-            const uint32_t o_addr = tmem_base + ((uint32_t)(q * 32) << 16) + O_COL + (uint32_t)(g2 * 32);
+            const uint32_t o_addr = tmem_base + ((uint32_t)(q * 32) << 16) + O_OFF + (uint32_t)(g2 * 32);
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj) {   // 16 channels at a time: O_0 and O_1 parts
                 uint32_t r0[16], r1[16];
                 nm_tmem_ld16(o_addr + (uint32_t)(jj * 16), r0);
-                nm_tmem_ld16(o_addr + (uint32_t)(HD + jj * 16), r1);
+                nm_tmem_ld16(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
                 nm_tmem_ld_wait();
                 uint32_t w[8];
 #pragma unroll
