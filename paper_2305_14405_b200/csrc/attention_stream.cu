@@ -37,8 +37,6 @@ constexpr int CK = 64;     // keys per chunk
 constexpr int ROWB = 128;  // bytes per tile row (64 x 16-bit)
 constexpr int STAGE = CK * ROWB;      // 8 KB
 constexpr int PBUF = BQ * ROWB;       // 16 KB
-constexpr int NTHREADS = 320;
-constexpr int NSOFT = 256;
 
 struct SArgs {
     int B, L, heads;
@@ -75,35 +73,38 @@ __device__ __forceinline__ float max3f(float a, float b, float c)
     return d;
 }
 
-template <typename T, bool CLAMP_HI>
-__global__ void __launch_bounds__(NTHREADS, 2)
+// NG = softmax groups per CTA: 2 (320 threads, 256 tensor-memory columns, two CTAs per SM) or
+// 1 (160 threads, 128 columns, three CTAs per SM: more tiles in flight per SM, fewer warps per tile).
+template <typename T, bool CLAMP_HI, int NG>
+__global__ void __launch_bounds__(160 * NG, NG == 1 ? 3 : 2)
 attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const SArgs a)
 {
     constexpr uint32_t IDESC_QK = nm_idesc(1, AT<T>::fmt, 0, 0, BQ, CK);   // S chunk: 128 x 64
     constexpr uint32_t IDESC_PV = nm_idesc(1, AT<T>::fmt, 0, 1, BQ, HD);   // O: 128 x 64, V MN-major
     constexpr uint32_t IDESC_QK1 = nm_idesc(1, AT<T>::fmt, 0, 0, BQ, 2 * CK);   // sweep 1: 128 x 128
-    constexpr uint32_t TMEM_COLS = 256;   // S0 | O0 | S1 | O1; sweep 1 writes 128 keys over [S_g | O_g]
+    constexpr uint32_t TMEM_COLS = 128 * NG;   // S0 | O0 (| S1 | O1); sweep 1 writes 128 keys over [S_g | O_g]
+    constexpr int NSOFT = 128 * NG;            // softmax threads
     constexpr uint32_t GRP_COLS = 128;    // tensor-memory columns of a group
     constexpr uint32_t O_OFF = 64;        // O_g within the group's columns
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bar_q, bar_drain[2];
-    __shared__ uint64_t bar_k_full[2][2], bar_k1_full[2][2], bar_v_full[2], bar_s_full[2], bar_p_empty[2];
+    __shared__ uint64_t bar_q, bar_drain[NG];
+    __shared__ uint64_t bar_k_full[NG][2], bar_k1_full[NG][2], bar_v_full[NG], bar_s_full[NG], bar_p_empty[NG];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float s_red[2][BQ];
+    __shared__ float s_red[NG][BQ];
 
     const int L = a.L;
     const int n = L / CK;      // chunks (even: L is a multiple of 128)
-    const int half = n >> 1;   // chunks per group in sweep 2
-    const int n128 = L / (2 * CK);   // 128-key chunks of sweep 1: group g takes g, g+2, ...
+    const int half = n / NG;   // chunks per group in sweep 2: group g takes g, g+NG, ...
+    const int n128 = L / (2 * CK);   // 128-key chunks of sweep 1: group g takes g, g+NG, ...
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* q_s = base;                       // 16 KB
     uint8_t* k_st = q_s + BQ * ROWB;           // [group][2] x 8 KB
-    uint8_t* v_st = k_st + 4 * STAGE;          // [group] x 8 KB
-    uint8_t* p_s = v_st + 2 * STAGE;           // [group] x 16 KB
-    float2* rep = reinterpret_cast<float2*>(p_s + 2 * PBUF);   // (n_exp + 1) x 16 copies
+    uint8_t* v_st = k_st + NG * 2 * STAGE;     // [group] x 8 KB
+    uint8_t* p_s = v_st + NG * STAGE;          // [group] x 16 KB
+    float2* rep = reinterpret_cast<float2*>(p_s + NG * PBUF);   // (n_exp + 1) x 16 copies
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int blocks_per_seq = L / BQ;
@@ -117,7 +118,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         nm_prefetch_tmap(&tmK);
         nm_prefetch_tmap(&tmV);
         nm_mbar_init(&bar_q, 1);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < NG; ++i) {
             nm_mbar_init(&bar_drain[i], 1);
             nm_mbar_init(&bar_k_full[i][0], 1);
             nm_mbar_init(&bar_k_full[i][1], 1);
@@ -135,9 +136,9 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         nm_grid_dependency_wait();   // Q, K, V come from the previous kernel
         nm_mbar_expect_tx(&bar_q, BQ * ROWB);
         nm_tma_load_3d(q_s, &tmQ, g * HD, qb * BQ, b, &bar_q);
-        for (int gi = 0; gi < 2; ++gi) {
+        for (int gi = 0; gi < NG; ++gi) {
             for (int st = 0; st < 2; ++st) {
-                const int c128 = gi + 2 * st;
+                const int c128 = gi + NG * st;
                 if (c128 >= n128) break;
                 uint8_t* dst = st == 0 ? k_st + (size_t)gi * 2 * STAGE : p_s + (size_t)gi * PBUF;
                 nm_mbar_expect_tx(&bar_k1_full[gi][st], 2 * STAGE);
@@ -148,16 +149,16 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             nm_tma_load_3d(v_st + (size_t)gi * STAGE, &tmV, g * HD, gi * CK, b, &bar_v_full[gi]);
         }
     }
-    if (warp == 1) {
+    if (warp == NG - 1) {
         nm_tmem_alloc(&tmem_slot, TMEM_COLS);
         nm_tmem_relinquish();
     }
-    if (warp >= 2) {
+    if (warp >= NG) {
         // 16-way replicated exp table: entry s, copy c at rep[s*16 + c].  A 64-bit warp load is served
         // half a warp at a time, so 16 copies already make arbitrary lookups conflict-free.  One extra
         // entry (a copy of the last) lets input 0 of a table whose range ends at 0 go unclamped.
         const int ne = a.n_exp;
-        for (int i = threadIdx.x - 64; i < (ne + 1) * 16; i += NSOFT) rep[i] = a.t_exp->kb[min(i >> 4, ne - 1)];
+        for (int i = threadIdx.x - 32 * NG; i < (ne + 1) * 16; i += NSOFT) rep[i] = a.t_exp->kb[min(i >> 4, ne - 1)];
     }
     nm_tc_fence_before();
     __syncthreads();
@@ -167,7 +168,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     nm_grid_launch_dependents();   // the next kernel may start its set-up
     nm_grid_dependency_wait();     // Q, K, V come from the previous kernel
 
-    if (warp < 2) {
+    if (warp < NG) {
         // ------------------------------------------------ control warp of group `warp`
         // Runs with all 32 lanes (barrier tests, counters and descriptors stay warp-uniform); one
         // elected lane issues the TMA and tcgen05 instructions.  It sleeps in a named barrier until
@@ -175,9 +176,9 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         //   S-consumed(i): chunk i's scores are in registers -> K stage i & 1 is free (load the chunk
         //                  after next into it) and S is free (issue Q K^T for the next chunk);
         //   P-ready(j):    the bf16 P tile of the j-th chunk of sweep 2 is in shared memory -> O += P V.
-        const int gi = warp;
+        const int gi = NG == 1 ? 0 : warp;
         const uint32_t bar_sc = 2 + 2 * gi, bar_pr = 3 + 2 * gi;
-        const int cnt1 = (n128 - gi + 1) >> 1;   // the group's 128-key chunks in sweep 1
+        const int cnt1 = (n128 - gi + NG - 1) / NG;   // the group's 128-key chunks in sweep 1
         uint8_t* my_k = k_st + (size_t)gi * 2 * STAGE;
         uint8_t* my_v = v_st + (size_t)gi * STAGE;
         uint8_t* my_p = p_s + (size_t)gi * PBUF;
@@ -207,18 +208,18 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             if (i + 1 < cnt1) issue_qk1(i + 1);
             if (ok && i + 2 < cnt1 && nm_elect_one()) {   // its MMAs are complete: the stage takes the chunk after next
                 uint8_t* dst = (i & 1) ? my_p : my_k;
-                const int key0 = (gi + 2 * (i + 2)) * 2 * CK;
+                const int key0 = (gi + NG * (i + 2)) * 2 * CK;
                 nm_mbar_expect_tx(&bar_k1_full[gi][i & 1], 2 * STAGE);
                 nm_tma_load_3d(dst, &tmK, g * HD, key0, b, &bar_k1_full[gi][i & 1]);
                 nm_tma_load_3d(dst + STAGE, &tmK, g * HD, key0 + CK, b, &bar_k1_full[gi][i & 1]);
             }
             __syncwarp();
         }
-        // ---- sweep 2: the group's j-th chunk is the 64 keys of chunk g + 2j; K stage j & 1
+        // ---- sweep 2: the group's j-th chunk is the 64 keys of chunk g + NG*j; K stage j & 1
         auto load_k = [&](int j) {
             if (ok && nm_elect_one()) {
                 nm_mbar_expect_tx(&bar_k_full[gi][j & 1], STAGE);
-                nm_tma_load_3d(my_k + (size_t)(j & 1) * STAGE, &tmK, g * HD, (gi + 2 * j) * CK, b, &bar_k_full[gi][j & 1]);
+                nm_tma_load_3d(my_k + (size_t)(j & 1) * STAGE, &tmK, g * HD, (gi + NG * j) * CK, b, &bar_k_full[gi][j & 1]);
             }
             __syncwarp();
         };
@@ -260,7 +261,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (!wait(&bar_p_empty[gi], (uint32_t)(j & 1))) ok = false;
                 if (ok && nm_elect_one()) {
                     nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
-                    nm_tma_load_3d(my_v, &tmV, g * HD, (gi + 2 * (j + 1)) * CK, b, &bar_v_full[gi]);
+                    nm_tma_load_3d(my_v, &tmV, g * HD, (gi + NG * (j + 1)) * CK, b, &bar_v_full[gi]);
                 }
                 __syncwarp();
             }
@@ -280,11 +281,11 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         // buffer g, P buffer g and accumulator O_g, so the two groups form two independent pipelines.
         // A warp never blocks on its group: it signals the control warp with bar.arrive.
         const int q = warp & 3;
-        const int g2 = (warp - 2) >> 2;
+        const int g2 = NG == 1 ? 0 : (warp - NG) >> 2;
         const int row = q * 32 + lane;
         const uint32_t bar_sc = 2 + 2 * g2, bar_pr = 3 + 2 * g2;
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g2 * GRP_COLS;
-        const int cnt1 = (n128 - g2 + 1) >> 1;   // the group's 128-key chunks in sweep 1
+        const int cnt1 = (n128 - g2 + NG - 1) / NG;   // the group's 128-key chunks in sweep 1
         const float inv_h = a.t_exp->inv_h, off = a.t_exp->off, nm1 = (float)(a.n_exp - 1);
         // this lane's copy of the replicated table, with the constant of the index trick folded in:
         // (bits << 7) = 0xA0000000 + s*128 (mod 2^32) for bits = 0x4B400000 + s
@@ -329,10 +330,12 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
             }
         }
-        s_red[g2][row] = m;
-        asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-        m = fmaxf(s_red[0][row], s_red[1][row]);
-        asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+        if constexpr (NG == 2) {   // the two groups saw different keys of the row
+            s_red[g2][row] = m;
+            asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+            m = fmaxf(s_red[0][row], s_red[1][row]);
+            asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+        }
         const float neg_ms = -(m * a.scale);
         float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
         const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(g2 * PBUF + row * ROWB);
@@ -395,31 +398,41 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
             asm volatile("bar.arrive %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");
         }
-        s_red[g2][row] = (sum0 + sum1) + (sum2 + sum3);
-        asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-        const float sum = s_red[0][row] + s_red[1][row];
+        float sum = (sum0 + sum1) + (sum2 + sum3);
+        if constexpr (NG == 2) {
+            s_red[g2][row] = sum;
+            asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+            sum = s_red[0][row] + s_red[1][row];
+        }
         // ---- r = PWL_recip(sigma), then (O_0 + O_1) * r; each group stores 32 of the 64 channels
         const int sr = nm_pwl_index(sum, a.t_rcp->inv_h, a.t_rcp->off, (float)(a.t_rcp->n - 1));
         const float2 kbr = a.t_rcp->kb[sr];
         const float rinv = __fmaf_rn(kbr.x, sum, kbr.y);
-        wait_all(&bar_p_empty[0], (uint32_t)((half - 1) & 1));   // the last P V of either group has completed
-        wait_all(&bar_p_empty[1], (uint32_t)((half - 1) & 1));
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg)   // the last P V of every group has completed
+            wait_all(&bar_p_empty[gg], (uint32_t)((half - 1) & 1));
         if (ok) {
             nm_tc_fence_after();
+            constexpr int CH = HD / NG;   // channels this warp stores
             T* orow = reinterpret_cast<T*>(a.out) + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
-                      (size_t)g * HD + g2 * 32;
-            const uint32_t o_addr = tmem_base + ((uint32_t)(q * 32) << 16) + O_OFF + (uint32_t)(g2 * 32);
+                      (size_t)g * HD + g2 * CH;
+            const uint32_t o_addr = tmem_base + ((uint32_t)(q * 32) << 16) + O_OFF + (uint32_t)(g2 * CH);
 #pragma unroll
-            for (int jj = 0; jj < 2; ++jj) {   // 16 channels at a time: O_0 and O_1 parts
+            for (int jj = 0; jj < CH / 16; ++jj) {   // 16 channels at a time, summed over the groups' accumulators
                 uint32_t r0[16], r1[16];
                 nm_tmem_ld16(o_addr + (uint32_t)(jj * 16), r0);
-                nm_tmem_ld16(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
+                if constexpr (NG == 2) nm_tmem_ld16(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
                 nm_tmem_ld_wait();
                 uint32_t w[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    w[k] = AT<T>::pack((__uint_as_float(r0[2 * k]) + __uint_as_float(r1[2 * k])) * rinv,
-                                       (__uint_as_float(r0[2 * k + 1]) + __uint_as_float(r1[2 * k + 1])) * rinv);
+                for (int k = 0; k < 8; ++k) {
+                    float x0 = __uint_as_float(r0[2 * k]), x1 = __uint_as_float(r0[2 * k + 1]);
+                    if constexpr (NG == 2) {
+                        x0 += __uint_as_float(r1[2 * k]);
+                        x1 += __uint_as_float(r1[2 * k + 1]);
+                    }
+                    w[k] = AT<T>::pack(x0 * rinv, x1 * rinv);
+                }
                 reinterpret_cast<uint4*>(orow)[2 * jj] = make_uint4(w[0], w[1], w[2], w[3]);
                 reinterpret_cast<uint4*>(orow)[2 * jj + 1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
@@ -428,7 +441,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 
     nm_tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == NG - 1) {
         __syncwarp();
         nm_tc_fence_after();
         nm_tmem_dealloc(tmem_base, TMEM_COLS);
@@ -454,7 +467,7 @@ nm_status make_map(nm_ctx* ctx, CUtensorMap* m, const void* ptr, nm_dtype dt, co
     return r == CUDA_SUCCESS ? NM_OK : NM_ERR_CUDA;
 }
 
-template <typename T, bool CLAMP_HI>
+template <typename T, bool CLAMP_HI, int NG>
 nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
 {
     SArgs a;
@@ -464,14 +477,14 @@ nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
     a.out = d->out;
     a.status = ctx->d_status;
     a.n_exp = ctx->h_tables[d->exp_slot].n;
-    const size_t smem = (size_t)BQ * ROWB + 6 * (size_t)STAGE + 2 * (size_t)PBUF + (size_t)(a.n_exp + 1) * 16 * sizeof(float2) + 1024;
+    const size_t smem = (size_t)BQ * ROWB + NG * (3 * (size_t)STAGE + (size_t)PBUF) + (size_t)(a.n_exp + 1) * 16 * sizeof(float2) + 1024;
     if (smem > 227 * 1024 - 2048) return NM_ERR_UNSUPPORTED;   // an exp table too large to replicate
     CUtensorMap tmQ, tmK, tmV;
     nm_status s;
     if ((s = make_map(ctx, &tmQ, d->Q, d->dtype, d, BQ)) != NM_OK) return s;
     if ((s = make_map(ctx, &tmK, d->K, d->dtype, d, CK)) != NM_OK) return s;
     if ((s = make_map(ctx, &tmV, d->V, d->dtype, d, CK)) != NM_OK) return s;
-    auto kern = attention_stream_kernel<T, CLAMP_HI>;
+    auto kern = attention_stream_kernel<T, CLAMP_HI, NG>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return NM_ERR_CUDA;
     const int64_t grid = (int64_t)d->B * d->heads * (d->L / BQ);
@@ -479,7 +492,7 @@ nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(NTHREADS);
+    cfg.blockDim = dim3(160 * NG);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -508,7 +521,14 @@ nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStr
     if (!nm_attention_stream_supported(d)) return NM_ERR_UNSUPPORTED;
     // the softmax input is never positive: a table whose range reaches 0 needs no upper clamp
     const bool clamp_hi = ctx->h_tables[d->exp_slot].x_max < 0.0f;
+    // one group per CTA (three CTAs per SM) measures a few percent faster up to L = 512, two groups beyond
+    const int groups = ctx->attn_groups ? ctx->attn_groups : (d->L <= 512 ? 1 : 2);
+    if (groups == 1) {
+        if (d->dtype == NM_BF16)
+            return clamp_hi ? launch<__nv_bfloat16, true, 1>(ctx, d, st) : launch<__nv_bfloat16, false, 1>(ctx, d, st);
+        return clamp_hi ? launch<__half, true, 1>(ctx, d, st) : launch<__half, false, 1>(ctx, d, st);
+    }
     if (d->dtype == NM_BF16)
-        return clamp_hi ? launch<__nv_bfloat16, true>(ctx, d, st) : launch<__nv_bfloat16, false>(ctx, d, st);
-    return clamp_hi ? launch<__half, true>(ctx, d, st) : launch<__half, false>(ctx, d, st);
+        return clamp_hi ? launch<__nv_bfloat16, true, 2>(ctx, d, st) : launch<__nv_bfloat16, false, 2>(ctx, d, st);
+    return clamp_hi ? launch<__half, true, 2>(ctx, d, st) : launch<__half, false, 2>(ctx, d, st);
 }

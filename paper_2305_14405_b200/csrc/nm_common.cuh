@@ -45,6 +45,7 @@ struct nm_ctx {
     NmProfRecord* prof;        // NM_PROF_MAX records, host memory
     int pdl;                   // launch kernels with programmatic stream serialization (prologue overlap)
     int attn_resident;         // algo 0 prefers the attention kernel with the score block resident in TMEM
+    int attn_groups;           // softmax groups per CTA of the streaming attention kernel (1 or 2; 0 = pick)
 };
 
 // Brackets one kernel launch with events when profiling is on; counts the launch always.

@@ -58,6 +58,21 @@ def test_attention_bf16(nm, ctx, algo, B, L, h, d, qk):
     assert_close_bf16(got, ref, "attention bf16 %s" % algo)
 
 
+@pytest.mark.parametrize("groups", ["1", "2"])
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+@pytest.mark.parametrize("B,L,h", [(2, 128, 3), (1, 384, 2), (1, 640, 1)])
+def test_attention_stream_groups(nm, monkeypatch, groups, dtype, B, L, h):
+    """The streaming kernel with one and with two softmax groups per CTA (the library picks by
+    sequence length; NM_ATTN_GROUPS, read when a context is created, forces either)."""
+    monkeypatch.setenv("NM_ATTN_GROUPS", groups)
+    c = nm.Context(0)
+    try:
+        got, ref = run(nm, c, dtype, B, L, h, 64, nm.ALGO_TC, seed=17 + L, qk_scale=0.8)
+    finally:
+        c.close()
+    assert_close_bf16(got, ref, "attention %s, %s group(s), L=%d" % (dtype, groups, L))
+
+
 @pytest.mark.parametrize("n", [16, 256])
 def test_attention_bf16_segment_counts(nm, ctx, n):
     got, ref = run(nm, ctx, "bf16", 1, 128, 2, 64, nm.ALGO_AUTO, seed=3, n=n, qk_scale=0.6)
