@@ -1,6 +1,6 @@
 """Benchmark of the PWL forward pass on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c1|c4|c5] [--segments n]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c1|c4|c5|rows] [--segments n]
     python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
 
 Default workload c3: the 12-layer BERT-base-shaped PWL encoder (batch 32, seq 512), the
@@ -38,7 +38,7 @@ def parse_args():
     p.add_argument("--steps", type=int, default=100)
     p.add_argument("--warmup", type=int, default=10)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
+    p.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5", "rows"])
     p.add_argument("--segments", type=int, default=64)
     p.add_argument("--seed", type=int, default=0)
     p.add_argument("--batch", type=int, default=0, help="override the batch size (c5 only)")
@@ -326,7 +326,109 @@ class ResnetWorkload:
         return 1.0
 
 
+class RowsWorkload:
+    """rows: the HBM-bound row kernels on a tensor far larger than L2: PWL LayerNorm over [2^20, 768] bf16
+    followed by an element-wise PWL GELU over the result; unit = algorithmic GB (one read and one write
+    per element and kernel)."""
+    metric = "PWL row kernels GB/s"
+    unit = "GB/s"
+    dtype = "bf16"
+    H = 768
+
+    def __init__(self, args):
+        self.args = args
+        self.rows = (args.batch or 1024) * 1024
+        self.units_per_step = 2 * 2 * self.rows * self.H * 2 / 1e9   # two kernels, read + write, 2 bytes
+
+    def config(self, world):
+        return {"workload": "rows_layernorm_gelu_bf16", "rows": self.rows, "hidden": self.H, "pwl_segments": 64,
+                "seed": self.args.seed, "parallelism": "replicas" if world > 1 else "single",
+                "l2": "each tensor is %.2f GB, far beyond the 126 MB L2; no flush" % (self.rows * self.H * 2 / 1e9)}
+
+    def flops_per_step(self):
+        return 0.0
+
+    def _np_inputs(self, rows, seed):
+        import nm_inputs
+        x = nm_inputs.matrix((rows, self.H), seed, "bf16", 1.0)
+        g = nm_inputs.matrix((self.H,), seed + 1, "f32", 0.1) + 1.0
+        b = nm_inputs.matrix((self.H,), seed + 2, "f32", 0.1)
+        return x, g.astype("float32"), b.astype("float32")
+
+    def setup(self, ctx, dev, rank):
+        import torch
+        import paper_2305_14405_b200 as nm
+        ctx.load_function_table(nm.SLOT_RSQRT, nm.FUNC_RSQRT, 64, 0.05, 8.0)
+        ctx.load_function_table(nm.SLOT_GELU, nm.FUNC_GELU, 64, -8.0, 8.0)
+        self.nm = nm
+        # one seeded 2^16-row block, tiled: the kernels' time does not depend on the values
+        xb, g, b = self._np_inputs(1 << 16, self.args.seed + rank)
+        blk = torch.from_numpy(xb).to(dev).bfloat16()
+        self.x = blk.repeat(self.rows // (1 << 16), 1).contiguous()
+        self.g = torch.from_numpy(g).to(dev)
+        self.b = torch.from_numpy(b).to(dev)
+        self.y = torch.empty_like(self.x)
+        self.z = torch.empty_like(self.x)
+        # end to end on a 2^16-row slice (100 MB each way) so that the default run stays short
+        self.e2e_rows = 1 << 16
+        self.xh = torch.from_numpy(xb).bfloat16().pin_memory()
+        self.zh = torch.empty_like(self.xh).pin_memory()
+        self.ctx = ctx
+        self.h2d = self.d2h = self.e2e_rows * self.H * 2
+        self.e2e_units = 2 * 2 * self.e2e_rows * self.H * 2 / 1e9
+
+    def step(self):
+        self.ctx.layernorm_pwl(self.x, self.g, self.b, self.y)
+        self.ctx.pwl_apply(self.nm.SLOT_GELU, self.y, self.z)
+
+    def host_step(self):
+        import torch
+        n = self.e2e_rows
+        self.x[:n].copy_(self.xh, non_blocking=True)
+        self.ctx.layernorm_pwl(self.x[:n], self.g, self.b, self.y[:n])
+        self.ctx.pwl_apply(self.nm.SLOT_GELU, self.y[:n], self.z[:n])
+        self.zh.copy_(self.z[:n], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    def roofline(self, prof, peaks, peak_kind):
+        out = {}
+        for kind in ("layernorm", "pwl_apply"):
+            n_k, ms_k, work_k = prof[kind]
+            gbs = work_k / (ms_k * 1e-3) / 1e9 if ms_k > 0 else 0.0
+            out[kind] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "avg_launch_us": ms_k / max(n_k, 1) * 1e3,
+                         "peak_source": "%s (HBM copy)" % peak_kind}
+        main = dict(out["layernorm"], kernel="layernorm")
+        return main, {"pwl_apply": out["pwl_apply"]}
+
+    def _oracle_run(self, rows):
+        import oracle
+        x, g, b = self._np_inputs(rows, self.args.seed)
+        t_r = oracle.Table.secant(oracle.RSQRT, 64, 0.05, 8.0)
+        t_g = oracle.Table.secant(oracle.GELU, 64, -8.0, 8.0)
+        t0 = time.perf_counter()
+        y = oracle.layernorm(x, g, b, 1e-5, t_r)
+        oracle.pwl_eval(t_g, y)
+        return time.perf_counter() - t0, oracle.num_threads()
+
+    def cpu_baseline(self):
+        t1, cores = self._oracle_run(1 << 12)
+        rows = int(max(1 << 12, min(self.rows, (1 << 12) * 15.0 / max(t1, 1e-4))))
+        secs, cores = self._oracle_run(rows)
+        return {"value": 2 * 2 * rows * self.H * 2 / 1e9 / secs, "unit": self.unit, "cores": cores, "kind": "oracle",
+                "sample": "%d of %d rows through both kernels, %.1f s" % (rows, self.rows, secs)}
+
+    def reference_setup(self):
+        self.ref_sample = "%d of %d rows through both kernels per step" % (1 << 14, self.rows)
+
+    def reference_step(self):
+        self._oracle_run(1 << 14)
+        return 2 * 2 * (1 << 14) * self.H * 2 / 1e9
+
+
 def make_workload(args):
+    if args.workload == "rows":
+        return RowsWorkload(args)
     return ResnetWorkload(args) if args.workload == "c5" else EncoderWorkload(args)
 
 
@@ -463,12 +565,14 @@ def main():
             if n_a:
                 tf = work_a / (ms_a * 1e-3) / 1e12
                 extra[kind] = {"bound": "alu", "achieved_tensor_tflops": tf, "avg_launch_us": ms_a / n_a * 1e3}
+        if hasattr(wl, "roofline"):   # a workload whose dominant kernel is not a GEMM brings its own
+            roofline, extra = wl.roofline(prof, peaks, peak_kind)
         line = {
             "metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config(world),
             "clocks": sampler.summary(),
-            "e2e": {"value": world * wl.units_per_step / (e2e_ms * 1e-3), "unit": wl.unit,
+            "e2e": {"value": world * getattr(wl, "e2e_units", wl.units_per_step) / (e2e_ms * 1e-3), "unit": wl.unit,
                     "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": e2e_ms},
             "gpu_launches": launches,
             "roofline": roofline,
