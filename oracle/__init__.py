@@ -243,6 +243,18 @@ def layernorm(z, gamma, beta, eps, t_rsqrt: Table):
     return y
 
 
+def layernorm_sqrt_recip(z, gamma, beta, eps, t_sqrt: Table, t_recip: Table):
+    """LayerNorm with r = PWLrecip(PWLsqrt(v + eps)): Section 3.2.2's sqrt(x) and 1/x tables."""
+    z = _f64(z)
+    rows, H = z.shape
+    g = _f64(gamma)
+    be = _f64(beta)
+    y = np.empty_like(z)
+    lib().nmo_layernorm_sqrt_recip(_dp(z), _dp(g), _dp(be), C.c_int64(rows), C.c_int32(H), C.c_double(eps),
+                                   t_sqrt.ref, t_recip.ref, _dp(y))
+    return y
+
+
 WEIGHT_NAMES = ("Wqkv", "bqkv", "Wo", "bo", "g1", "be1", "W1", "b1", "W2", "b2", "g2", "be2")
 
 

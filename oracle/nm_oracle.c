@@ -20,7 +20,7 @@
  *                       the range reuse the first / last segment's k and b).
  *   nmo_linear          Section 3.1: a linear operator is a matrix product
  *                       plus matrix adds.
- *   nmo_attention, nmo_layernorm, nmo_encoder_layer
+ *   nmo_attention, nmo_layernorm, nmo_layernorm_sqrt_recip, nmo_encoder_layer
  *                       the BERT encoder layer of Section 5 with exp, 1/x,
  *                       rsqrt and GELU replaced by PWL tables.
  *   nmo_linear_i8       the INT8 evaluation of Section 5: exact integer
@@ -329,6 +329,27 @@ void nmo_layernorm(const double* z, const double* gamma, const double* beta,
         for (int c = 0; c < H; ++c) v += (zr[c] - mu) * (zr[c] - mu);
         v /= (double)H;
         double r = pwl_one(t_rsqrt, v + eps, NULL);
+        for (int c = 0; c < H; ++c) y[r0 * H + c] = (zr[c] - mu) * r * gamma[c] + beta[c];
+    }
+}
+
+/* The same LayerNorm with the reciprocal square root taken as the paper's own two
+ * functions (Section 3.2.2 lists sqrt(x) and 1/x): r = PWLrecip(PWLsqrt(v + eps)). */
+void nmo_layernorm_sqrt_recip(const double* z, const double* gamma, const double* beta,
+                              int64_t rows, int32_t H, double eps, const nmo_pwl* t_sqrt,
+                              const nmo_pwl* t_recip, double* y)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t r0 = 0; r0 < rows; ++r0) {
+        const double* zr = z + r0 * H;
+        double mu = 0.0;
+        for (int c = 0; c < H; ++c) mu += zr[c];
+        mu /= (double)H;
+        double v = 0.0;
+        for (int c = 0; c < H; ++c) v += (zr[c] - mu) * (zr[c] - mu);
+        v /= (double)H;
+        double sd = pwl_one(t_sqrt, v + eps, NULL);
+        double r = pwl_one(t_recip, sd, NULL);
         for (int c = 0; c < H; ++c) y[r0 * H + c] = (zr[c] - mu) * r * gamma[c] + beta[c];
     }
 }

@@ -300,6 +300,50 @@ def test_layernorm_pwl_uses_table_on_variance_plus_eps():
     assert np.allclose(y.std(axis=1), np.sqrt(v) * r, rtol=1e-12)
 
 
+def test_layernorm_sqrt_recip_exact_mode_is_library_layer_norm():
+    """With both tables exact, 1/sqrt(v + eps) is recovered and the result is the textbook LayerNorm."""
+    rng = np.random.default_rng(15)
+    z = rng.standard_normal((7, 40)) * 2 - 0.5
+    g = rng.standard_normal(40)
+    b = rng.standard_normal(40)
+    y = oracle.layernorm_sqrt_recip(z, g, b, 1e-5, Table.exact(oracle.SQRT), Table.exact(oracle.RECIP))
+    ref = torch.nn.functional.layer_norm(torch.from_numpy(z), (40,), torch.from_numpy(g), torch.from_numpy(b), 1e-5)
+    assert np.allclose(y, ref.numpy(), rtol=1e-11, atol=1e-12)
+
+
+def test_layernorm_sqrt_recip_composes_the_two_tables_in_that_order():
+    """r = recip_table(sqrt_table(v + eps)): checked through the row statistics of the output (gamma 1,
+    beta 0: zero mean, standard deviation sqrt(v) * r), and against the swapped order, which differs."""
+    rng = np.random.default_rng(16)
+    z = rng.standard_normal((6, 64)) * np.array([[0.6], [0.9], [1.2], [1.5], [1.8], [2.1]])
+    ts = Table.secant(oracle.SQRT, 16, 0.0625, 9.0)
+    tr = Table.secant(oracle.RECIP, 16, 0.25, 3.0)
+    y = oracle.layernorm_sqrt_recip(z, np.ones(64), np.zeros(64), 1e-5, ts, tr)
+    assert np.abs(y.mean(axis=1)).max() < 1e-14
+    v = z.var(axis=1)
+    r = tr(ts(v + 1e-5))
+    assert np.allclose(y.std(axis=1), np.sqrt(v) * r, rtol=1e-12)
+    swapped = ts(tr(v + 1e-5))
+    assert np.abs(swapped - r).max() > 1e-3
+
+
+def test_layernorm_sqrt_recip_error_against_exact_is_within_the_secant_bounds():
+    """|recip_t(sqrt_t(u)) - u^-1/2| <= e_r + e_s / s_min^2 with the secant-line bounds e = h^2/8 max|f''|
+    (sqrt: |f''| = u^-3/2 / 4; 1/x: |f''| = 2 / x^3) and 1/x having slope at most 1/s_min^2."""
+    a, b, n = 0.25, 9.0, 64
+    sa, sb = 0.45, 3.05   # range of the sqrt table's values with margin for its error
+    ts = Table.secant(oracle.SQRT, n, a, b)
+    tr = Table.secant(oracle.RECIP, n, sa, sb)
+    u = np.linspace(a, b, 20001)
+    got = tr(ts(u))
+    e_s = ((b - a) / n) ** 2 / 8 * (a ** -1.5 / 4)
+    e_r = ((sb - sa) / n) ** 2 / 8 * (2 / sa ** 3)
+    bound = e_r + e_s / sa ** 2
+    err = np.abs(got - u ** -0.5)
+    assert err.max() <= bound * (1 + 1e-6)
+    assert err.max() > bound / 50   # the bound is not vacuous
+
+
 # ---------------------------------------------------------------- encoder layer --
 
 def _torch_encoder_layer(x, w, B, L, h):
