@@ -42,6 +42,8 @@ def parse_args():
     p.add_argument("--segments", type=int, default=64)
     p.add_argument("--seed", type=int, default=0)
     p.add_argument("--batch", type=int, default=0, help="override the batch size (c5 only)")
+    p.add_argument("--ln-two-table", action="store_true",
+                   help="rows workload: LayerNorm as PWL_recip(PWL_sqrt(v + eps)) instead of one rsqrt table")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--algo", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     return p.parse_args()
@@ -342,6 +344,7 @@ class RowsWorkload:
 
     def config(self, world):
         return {"workload": "rows_layernorm_gelu_bf16", "rows": self.rows, "hidden": self.H, "pwl_segments": 64,
+                "layernorm": "sqrt table then 1/x table" if self.args.ln_two_table else "one rsqrt table",
                 "seed": self.args.seed, "parallelism": "replicas" if world > 1 else "single",
                 "l2": "each tensor is %.2f GB, far beyond the 126 MB L2; no flush" % (self.rows * self.H * 2 / 1e9)}
 
@@ -360,6 +363,8 @@ class RowsWorkload:
         import paper_2305_14405_b200 as nm
         ctx.load_function_table(nm.SLOT_RSQRT, nm.FUNC_RSQRT, 64, 0.05, 8.0)
         ctx.load_function_table(nm.SLOT_GELU, nm.FUNC_GELU, 64, -8.0, 8.0)
+        ctx.load_function_table(nm.SLOT_USER0, nm.FUNC_SQRT, 64, 0.05, 8.0)
+        ctx.load_function_table(nm.SLOT_USER0 + 1, nm.FUNC_RECIP, 64, 0.2, 3.0)
         self.nm = nm
         # one seeded 2^16-row block, tiled: the kernels' time does not depend on the values
         xb, g, b = self._np_inputs(1 << 16, self.args.seed + rank)
@@ -377,15 +382,21 @@ class RowsWorkload:
         self.h2d = self.d2h = self.e2e_rows * self.H * 2
         self.e2e_units = 2 * 2 * self.e2e_rows * self.H * 2 / 1e9
 
+    def _ln(self, x, y):
+        if self.args.ln_two_table:
+            self.ctx.layernorm_pwl_sqrt_recip(x, self.g, self.b, y, self.nm.SLOT_USER0, self.nm.SLOT_USER0 + 1)
+        else:
+            self.ctx.layernorm_pwl(x, self.g, self.b, y)
+
     def step(self):
-        self.ctx.layernorm_pwl(self.x, self.g, self.b, self.y)
+        self._ln(self.x, self.y)
         self.ctx.pwl_apply(self.nm.SLOT_GELU, self.y, self.z)
 
     def host_step(self):
         import torch
         n = self.e2e_rows
         self.x[:n].copy_(self.xh, non_blocking=True)
-        self.ctx.layernorm_pwl(self.x[:n], self.g, self.b, self.y[:n])
+        self._ln(self.x[:n], self.y[:n])
         self.ctx.pwl_apply(self.nm.SLOT_GELU, self.y[:n], self.z[:n])
         self.zh.copy_(self.z[:n], non_blocking=True)
         torch.cuda.current_stream().synchronize()
@@ -405,9 +416,14 @@ class RowsWorkload:
         import oracle
         x, g, b = self._np_inputs(rows, self.args.seed)
         t_r = oracle.Table.secant(oracle.RSQRT, 64, 0.05, 8.0)
+        t_s = oracle.Table.secant(oracle.SQRT, 64, 0.05, 8.0)
+        t_i = oracle.Table.secant(oracle.RECIP, 64, 0.2, 3.0)
         t_g = oracle.Table.secant(oracle.GELU, 64, -8.0, 8.0)
         t0 = time.perf_counter()
-        y = oracle.layernorm(x, g, b, 1e-5, t_r)
+        if self.args.ln_two_table:
+            y = oracle.layernorm_sqrt_recip(x, g, b, 1e-5, t_s, t_i)
+        else:
+            y = oracle.layernorm(x, g, b, 1e-5, t_r)
         oracle.pwl_eval(t_g, y)
         return time.perf_counter() - t0, oracle.num_threads()
 

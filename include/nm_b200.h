@@ -201,6 +201,16 @@ nm_status nm_layernorm_pwl(nm_ctx* ctx, const void* x, const float* gamma, const
                            int64_t rows, int32_t H, float eps, int32_t rsqrt_slot, nm_dtype dtype,
                            void* stream);
 
+/* The same LayerNorm with the reciprocal square root taken as the two functions Section 3.2.2
+ * itself lists, sqrt(x) and 1/x, one table each:
+ *     r = PWL_recip(PWL_sqrt(v + eps))
+ * sqrt_slot holds a table over the range of v + eps, recip_slot one over the range of its square
+ * root (not the attention's 1/x table, whose range is that of the softmax row sums).  Arguments,
+ * layout and errors as for nm_layernorm_pwl; NM_ERR_NO_TABLE if either slot is empty. */
+nm_status nm_layernorm_pwl_sqrt_recip(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
+                                      int64_t rows, int32_t H, float eps, int32_t sqrt_slot, int32_t recip_slot,
+                                      nm_dtype dtype, void* stream);
+
 /* Symmetric int8 quantisation of an activation tensor with a static scale:
  * q[i] = clamp(rint(x[i] * inv_scale), -127, 127), ties to even (the INT8
  * evaluation of Section 5).  x: device, `count` elements of dtype; q: device int8. */

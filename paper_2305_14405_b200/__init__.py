@@ -26,7 +26,7 @@ STATIC_WS_BYTES = 32 << 20
 EXPORTS = [
     "nm_status_string", "nm_ctx_create", "nm_ctx_destroy", "nm_ctx_poll_status", "nm_ctx_launch_count",
     "nm_pwl_table_build", "nm_pwl_table_load", "nm_pwl_apply", "nm_linear_pwl", "nm_attention_pwl",
-    "nm_layernorm_pwl", "nm_quantize_i8", "nm_encoder_workspace_bytes", "nm_encoder_layer", "nm_encoder_stack",
+    "nm_layernorm_pwl", "nm_layernorm_pwl_sqrt_recip", "nm_quantize_i8", "nm_encoder_workspace_bytes", "nm_encoder_layer", "nm_encoder_stack",
     "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
     "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
     "nm_resnet50_forward", "nm_resnet50_forward_host", "nm_pwl_table_build_elastic",
@@ -121,6 +121,8 @@ def load():
     lib.nm_attention_pwl.argtypes = [C.c_void_p, C.POINTER(AttnDesc), C.c_void_p]
     lib.nm_layernorm_pwl.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                      C.c_int32, C.c_float, C.c_int32, C.c_int, C.c_void_p]
+    lib.nm_layernorm_pwl_sqrt_recip.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                                C.c_int32, C.c_float, C.c_int32, C.c_int32, C.c_int, C.c_void_p]
     lib.nm_quantize_i8.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_void_p, C.c_void_p]
     lib.nm_encoder_workspace_bytes.restype = C.c_size_t
     lib.nm_encoder_workspace_bytes.argtypes = [C.POINTER(EncoderCfg)]
@@ -320,6 +322,12 @@ class Context:
         rows, H = x.shape
         _check(self._lib.nm_layernorm_pwl(self._h, _ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), rows, H, eps,
                                           rsqrt_slot, dtype_of(x), _stream(stream)), "nm_layernorm_pwl")
+
+    def layernorm_pwl_sqrt_recip(self, x, gamma, beta, y, sqrt_slot, recip_slot, eps=1e-5, stream=None):
+        rows, H = x.shape
+        _check(self._lib.nm_layernorm_pwl_sqrt_recip(self._h, _ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), rows, H,
+                                                     eps, sqrt_slot, recip_slot, dtype_of(x), _stream(stream)),
+               "nm_layernorm_pwl_sqrt_recip")
 
     def quantize_i8(self, x, inv_scale, q, stream=None):
         _check(self._lib.nm_quantize_i8(self._h, _ptr(x), dtype_of(x), x.numel(), inv_scale, _ptr(q),

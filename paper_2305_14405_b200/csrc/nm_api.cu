@@ -359,7 +359,24 @@ nm_status nm_layernorm_pwl(nm_ctx* ctx, const void* x, const float* gamma, const
     if (!x || !y || !gamma || !beta) return NM_ERR_INVALID_ARG;
     if (H % 8 != 0) return NM_ERR_SHAPE;
     if (!nm_aligned16(x) || !nm_aligned16(y) || !nm_aligned16(gamma) || !nm_aligned16(beta)) return NM_ERR_ALIGNMENT;
-    return nm_launch_layernorm(ctx, x, gamma, beta, y, rows, H, eps, rsqrt_slot, dtype, (cudaStream_t)stream);
+    return nm_launch_layernorm(ctx, x, gamma, beta, y, rows, H, eps, rsqrt_slot, NM_SLOT_NONE, dtype, (cudaStream_t)stream);
+}
+
+nm_status nm_layernorm_pwl_sqrt_recip(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
+                                      int64_t rows, int32_t H, float eps, int32_t sqrt_slot, int32_t recip_slot,
+                                      nm_dtype dtype, void* stream)
+{
+    if (!ctx) return NM_ERR_INVALID_ARG;
+    if (rows < 0 || H < 0) return NM_ERR_SHAPE;
+    nm_status s = need_table(ctx, sqrt_slot);
+    if (s != NM_OK) return s;
+    s = need_table(ctx, recip_slot);
+    if (s != NM_OK) return s;
+    if (rows == 0 || H == 0) return NM_OK;
+    if (!x || !y || !gamma || !beta) return NM_ERR_INVALID_ARG;
+    if (H % 8 != 0) return NM_ERR_SHAPE;
+    if (!nm_aligned16(x) || !nm_aligned16(y) || !nm_aligned16(gamma) || !nm_aligned16(beta)) return NM_ERR_ALIGNMENT;
+    return nm_launch_layernorm(ctx, x, gamma, beta, y, rows, H, eps, sqrt_slot, recip_slot, dtype, (cudaStream_t)stream);
 }
 
 nm_status nm_selftest_bounded_wait(nm_ctx* ctx, int64_t limit_cycles, void* stream)

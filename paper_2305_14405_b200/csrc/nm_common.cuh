@@ -594,7 +594,8 @@ static inline size_t nm_dtype_size(nm_dtype t)
 nm_status nm_launch_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int64_t count, nm_dtype dtype,
                               int32_t* idx_out, cudaStream_t st);
 nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
-                              int64_t rows, int32_t H, float eps, int32_t slot, nm_dtype dtype, cudaStream_t st);
+                              int64_t rows, int32_t H, float eps, int32_t slot, int32_t slot2, nm_dtype dtype,
+                              cudaStream_t st);   // slot2 != NM_SLOT_NONE: sqrt in slot, 1/x in slot2
 nm_status nm_launch_wait_selftest(nm_ctx* ctx, long long limit_cycles, cudaStream_t st);
 nm_status nm_launch_quantize(nm_ctx* ctx, const void* x, nm_dtype dtype, int64_t count, float inv_scale,
                              int8_t* q, cudaStream_t st);

@@ -76,7 +76,8 @@ __global__ void __launch_bounds__(256) pwl_apply_kernel(const NmTable* __restric
 // ---- LayerNorm with PWL rsqrt: one warp per row, the row kept in registers ------
 //   mu = mean(z); v = mean((z-mu)^2); r = PWL_rsqrt(v + eps); y = (z-mu)*r*gamma + beta
 template <typename T, int ITERS>
-__global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restrict__ tab, const T* __restrict__ x,
+__global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restrict__ tab,
+                                                        const NmTable* __restrict__ tab2, const T* __restrict__ x,
                                                         const float* __restrict__ gamma,
                                                         const float* __restrict__ beta, T* __restrict__ y,
                                                         int64_t rows, int H, float eps)
@@ -144,7 +145,12 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restric
         const float var = sq / (float)H + eps;
         const int s = nm_pwl_index(var, inv_h, off, nm1);
         const float2 kb = tab->kb[s];
-        const float r = __fmaf_rn(kb.x, var, kb.y);
+        float r = __fmaf_rn(kb.x, var, kb.y);
+        if (tab2) {   // two-table form: `tab` gave sqrt(v + eps), `tab2` takes its reciprocal
+            const int s2 = nm_pwl_index(r, tab2->inv_h, tab2->off, (float)(tab2->n - 1));
+            const float2 kb2 = tab2->kb[s2];
+            r = __fmaf_rn(kb2.x, r, kb2.y);
+        }
         T* yr = y + row * H;
 #pragma unroll
         for (int it = 0; it < ITERS; ++it) {
@@ -210,7 +216,7 @@ __global__ void wait_selftest_kernel(int* status, long long limit_cycles, int* r
 }
 
 template <typename T>
-nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const void* x, const float* gamma, const float* beta, void* y,
+nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const NmTable* tab2, const void* x, const float* gamma, const float* beta, void* y,
                     int64_t rows, int H, float eps, cudaStream_t st)
 {
     constexpr int N = VecOf<T>::N;
@@ -233,7 +239,7 @@ nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const void* x, const float*
     cfg.numAttrs = ctx->pdl ? 1 : 0;
     const T* xt = (const T*)x;
     T* yt = (T*)y;
-#define NM_LN_CASE(I) cudaLaunchKernelEx(&cfg, layernorm_kernel<T, I>, tab, xt, gamma, beta, yt, rows, H, eps)
+#define NM_LN_CASE(I) cudaLaunchKernelEx(&cfg, layernorm_kernel<T, I>, tab, tab2, xt, gamma, beta, yt, rows, H, eps)
     if (iters <= 1) NM_LN_CASE(1);
     else if (iters <= 2) NM_LN_CASE(2);
     else if (iters <= 3) NM_LN_CASE(3);
@@ -277,13 +283,15 @@ nm_status nm_launch_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int
 }
 
 nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
-                              int64_t rows, int32_t H, float eps, int32_t slot, nm_dtype dtype, cudaStream_t st)
+                              int64_t rows, int32_t H, float eps, int32_t slot, int32_t slot2, nm_dtype dtype,
+                              cudaStream_t st)
 {
     const NmTable* tab = ctx->d_tables + slot;
+    const NmTable* tab2 = slot2 == NM_SLOT_NONE ? nullptr : ctx->d_tables + slot2;
     switch (dtype) {
-    case NM_F32: return launch_ln<float>(ctx, tab, x, gamma, beta, y, rows, H, eps, st);
-    case NM_BF16: return launch_ln<__nv_bfloat16>(ctx, tab, x, gamma, beta, y, rows, H, eps, st);
-    case NM_F16: return launch_ln<__half>(ctx, tab, x, gamma, beta, y, rows, H, eps, st);
+    case NM_F32: return launch_ln<float>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, st);
+    case NM_BF16: return launch_ln<__nv_bfloat16>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, st);
+    case NM_F16: return launch_ln<__half>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, st);
     default: return NM_ERR_UNSUPPORTED;
     }
 }

@@ -90,6 +90,39 @@ def test_layernorm_parity(nm, ctx, dtype, rows, H):
         assert_close_bf16(to_np(yd), ref, "layernorm " + dtype)
 
 
+@pytest.mark.parametrize("dtype,rows,H,n", [("f32", 96, 256, 64), ("bf16", 1024, 768, 64), ("bf16", 333, 1024, 16),
+                                            ("f16", 100, 768, 256), ("bf16", 5, 8, 64)])
+def test_layernorm_sqrt_recip_parity(nm, ctx, dtype, rows, H, n):
+    """LayerNorm in the paper's two-function form: sqrt table on v + eps, 1/x table on its result."""
+    import oracle as orc
+    rng = np.random.default_rng(rows * 3 + H)
+    z = nm_inputs.round_to((rng.standard_normal((rows, H)) * rng.uniform(0.6, 1.8, (rows, 1)) + 0.3).astype(np.float32), dtype)
+    g = (1 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    b = (0.1 * rng.standard_normal(H)).astype(np.float32)
+    r_sqrt, r_recip = (0.0625, 9.0), (0.2, 3.2)
+    tabs = {}
+    for slot, func, (lo, hi) in ((nm.SLOT_USER0, nm.FUNC_SQRT, r_sqrt), (nm.SLOT_USER0 + 1, nm.FUNC_RECIP, r_recip)):
+        k, bb = ctx.load_function_table(slot, func, n, lo, hi)
+        t = orc.Table.secant(func, n, lo, hi)
+        assert np.array_equal(np.asarray(k, np.float32), t.k) and np.array_equal(np.asarray(bb, np.float32), t.b)
+        tabs[func] = t
+    td = nm_inputs.torch_dtype(dtype)
+    zd = torch.from_numpy(z).cuda().to(td)
+    yd = torch.empty_like(zd)
+    ctx.layernorm_pwl_sqrt_recip(zd, torch.from_numpy(g).cuda(), torch.from_numpy(b).cuda(), yd, nm.SLOT_USER0,
+                                 nm.SLOT_USER0 + 1, eps=1e-5)
+    ref = orc.layernorm_sqrt_recip(z, g, b, 1e-5, tabs[nm.FUNC_SQRT], tabs[nm.FUNC_RECIP])
+    if dtype == "f32":
+        assert_close_f32(to_np(yd), ref, "layernorm sqrt+recip f32")
+    else:
+        assert_close_bf16(to_np(yd), ref, "layernorm sqrt+recip " + dtype)
+    # an empty slot is an error, not a silent fallback
+    with pytest.raises(nm.NmError) as ei:
+        ctx.layernorm_pwl_sqrt_recip(zd, torch.from_numpy(g).cuda(), torch.from_numpy(b).cuda(), yd, nm.SLOT_USER0,
+                                     13, eps=1e-5)   # slot 13 is never loaded in this module
+    assert ei.value.code == 4
+
+
 def test_layernorm_rejects_bad_shapes(nm, ctx):
     load_tables_both(ctx, 64, {"rsqrt": RANGES["rsqrt"]})
     z = torch.zeros(4, 12, device="cuda")
