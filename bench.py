@@ -44,6 +44,8 @@ def parse_args():
     p.add_argument("--batch", type=int, default=0, help="override the batch size (c5 only)")
     p.add_argument("--ln-two-table", action="store_true",
                    help="rows workload: LayerNorm as PWL_recip(PWL_sqrt(v + eps)) instead of one rsqrt table")
+    p.add_argument("--hidden", type=int, default=0, help="encoder workloads: override H (heads = H/64, F = 4H)")
+    p.add_argument("--layers", type=int, default=0, help="encoder workloads: override the number of layers")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--algo", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     return p.parse_args()
@@ -146,6 +148,11 @@ class EncoderWorkload:
         import nm_inputs
         self.args = args
         self.cfg = nm_inputs.with_(nm_inputs.CONFIGS[args.workload], segments=args.segments)
+        if args.hidden or args.layers:   # width / depth sweep: same recipe, other shape
+            H = args.hidden or self.cfg.H
+            assert H % 64 == 0, "--hidden must be a multiple of the head size 64"
+            self.cfg = nm_inputs.with_(self.cfg, H=H, heads=H // 64, F=4 * H, layers=args.layers or self.cfg.layers,
+                                       name="%s_H%d_L%d" % (self.cfg.name, H, args.layers or self.cfg.layers))
         self.dtype = self.cfg.dtype
         self.units_per_step = self.cfg.T
 
