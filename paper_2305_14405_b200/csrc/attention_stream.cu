@@ -46,11 +46,14 @@ struct SArgs {
     void* out;
     int* status;
     int n_exp;
+    int8_t* out_q;       // when set: the output goes out as int8 codes (of the value rounded to T) instead
+    float q_inv_scale;
 };
 
 template <typename T> struct AT;
 template <> struct AT<__nv_bfloat16> {
     static constexpr uint32_t fmt = 1;
+    static __device__ __forceinline__ float round(float a) { return __bfloat162float(__float2bfloat16_rn(a)); }
     static __device__ __forceinline__ uint32_t pack(float a, float b)
     {
         __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -59,6 +62,7 @@ template <> struct AT<__nv_bfloat16> {
 };
 template <> struct AT<__half> {
     static constexpr uint32_t fmt = 0;
+    static __device__ __forceinline__ float round(float a) { return __half2float(__float2half_rn(a)); }
     static __device__ __forceinline__ uint32_t pack(float a, float b)
     {
         __half2 h = __floats2half2_rn(a, b);
@@ -423,18 +427,27 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 nm_tmem_ld16(o_addr + (uint32_t)(jj * 16), r0);
                 if constexpr (NG == 2) nm_tmem_ld16(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
                 nm_tmem_ld_wait();
-                uint32_t w[8];
+                float v[16];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    float x0 = __uint_as_float(r0[2 * k]), x1 = __uint_as_float(r0[2 * k + 1]);
-                    if constexpr (NG == 2) {
-                        x0 += __uint_as_float(r1[2 * k]);
-                        x1 += __uint_as_float(r1[2 * k + 1]);
-                    }
-                    w[k] = AT<T>::pack(x0 * rinv, x1 * rinv);
+                for (int k = 0; k < 16; ++k) {
+                    float x = __uint_as_float(r0[k]);
+                    if constexpr (NG == 2) x += __uint_as_float(r1[k]);
+                    v[k] = x * rinv;
                 }
-                reinterpret_cast<uint4*>(orow)[2 * jj] = make_uint4(w[0], w[1], w[2], w[3]);
-                reinterpret_cast<uint4*>(orow)[2 * jj + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                if (a.out_q) {
+                    int8_t code[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) code[k] = nm_quant_i8(AT<T>::round(v[k]), a.q_inv_scale);
+                    int8_t* qrow = a.out_q + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
+                                   (size_t)g * HD + g2 * CH;
+                    reinterpret_cast<uint4*>(qrow)[jj] = *reinterpret_cast<const uint4*>(code);
+                } else {
+                    uint32_t w[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) w[k] = AT<T>::pack(v[2 * k], v[2 * k + 1]);
+                    reinterpret_cast<uint4*>(orow)[2 * jj] = make_uint4(w[0], w[1], w[2], w[3]);
+                    reinterpret_cast<uint4*>(orow)[2 * jj + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                }
             }
         }
     }
@@ -468,7 +481,7 @@ nm_status make_map(nm_ctx* ctx, CUtensorMap* m, const void* ptr, nm_dtype dt, co
 }
 
 template <typename T, bool CLAMP_HI, int NG>
-nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
+nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st, int8_t* out_q, float q_inv_scale)
 {
     SArgs a;
     a.B = d->B; a.L = d->L; a.heads = d->heads; a.scale = d->scale;
@@ -477,6 +490,8 @@ nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
     a.out = d->out;
     a.status = ctx->d_status;
     a.n_exp = ctx->h_tables[d->exp_slot].n;
+    a.out_q = out_q;
+    a.q_inv_scale = q_inv_scale;
     const size_t smem = (size_t)BQ * ROWB + NG * (3 * (size_t)STAGE + (size_t)PBUF) + (size_t)(a.n_exp + 1) * 16 * sizeof(float2) + 1024;
     if (smem > 227 * 1024 - 2048) return NM_ERR_UNSUPPORTED;   // an exp table too large to replicate
     CUtensorMap tmQ, tmK, tmV;
@@ -516,7 +531,8 @@ bool nm_attention_stream_supported(const nm_attn_desc* d)
     return true;
 }
 
-nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st)
+nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st, int8_t* out_q,
+                                     float q_inv_scale)
 {
     if (!nm_attention_stream_supported(d)) return NM_ERR_UNSUPPORTED;
     // the softmax input is never positive: a table whose range reaches 0 needs no upper clamp
@@ -525,10 +541,10 @@ nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStr
     const int groups = ctx->attn_groups ? ctx->attn_groups : (d->L <= 512 ? 1 : 2);
     if (groups == 1) {
         if (d->dtype == NM_BF16)
-            return clamp_hi ? launch<__nv_bfloat16, true, 1>(ctx, d, st) : launch<__nv_bfloat16, false, 1>(ctx, d, st);
-        return clamp_hi ? launch<__half, true, 1>(ctx, d, st) : launch<__half, false, 1>(ctx, d, st);
+            return clamp_hi ? launch<__nv_bfloat16, true, 1>(ctx, d, st, out_q, q_inv_scale) : launch<__nv_bfloat16, false, 1>(ctx, d, st, out_q, q_inv_scale);
+        return clamp_hi ? launch<__half, true, 1>(ctx, d, st, out_q, q_inv_scale) : launch<__half, false, 1>(ctx, d, st, out_q, q_inv_scale);
     }
     if (d->dtype == NM_BF16)
-        return clamp_hi ? launch<__nv_bfloat16, true, 2>(ctx, d, st) : launch<__nv_bfloat16, false, 2>(ctx, d, st);
-    return clamp_hi ? launch<__half, true, 2>(ctx, d, st) : launch<__half, false, 2>(ctx, d, st);
+        return clamp_hi ? launch<__nv_bfloat16, true, 2>(ctx, d, st, out_q, q_inv_scale) : launch<__nv_bfloat16, false, 2>(ctx, d, st, out_q, q_inv_scale);
+    return clamp_hi ? launch<__half, true, 2>(ctx, d, st, out_q, q_inv_scale) : launch<__half, false, 2>(ctx, d, st, out_q, q_inv_scale);
 }

@@ -316,8 +316,20 @@ nm_status nm_linear_pwl(nm_ctx* ctx, const nm_linear_desc* d, void* stream)
     return nm_launch_linear_simt(ctx, d, st);
 }
 
+// out_q != nullptr asks for the output as int8 codes in out_q instead of d->out; *fused tells whether the
+// kernel chosen could do that (the caller quantises d->out itself otherwise).
+static nm_status attention_dispatch(nm_ctx* ctx, const nm_attn_desc* d, void* stream, int8_t* out_q,
+                                    float q_inv_scale, bool* fused);
+
 nm_status nm_attention_pwl(nm_ctx* ctx, const nm_attn_desc* d, void* stream)
 {
+    return attention_dispatch(ctx, d, stream, nullptr, 0.f, nullptr);
+}
+
+static nm_status attention_dispatch(nm_ctx* ctx, const nm_attn_desc* d, void* stream, int8_t* out_q,
+                                    float q_inv_scale, bool* fused)
+{
+    if (fused) *fused = false;
     if (!ctx || !d) return NM_ERR_INVALID_ARG;
     if (d->B < 0 || d->L < 0 || d->heads < 0 || d->d < 0) return NM_ERR_SHAPE;
     nm_status s = need_table(ctx, d->exp_slot);
@@ -342,14 +354,19 @@ nm_status nm_attention_pwl(nm_ctx* ctx, const nm_attn_desc* d, void* stream)
     const bool tc = nm_attention_stream_supported(d);
     if (d->algo == 2) return tc ? nm_launch_attention_stream(ctx, d, st) : NM_ERR_UNSUPPORTED;
     if (tc) {
-        const nm_status s = nm_launch_attention_stream(ctx, d, st);
-        if (s != NM_ERR_UNSUPPORTED) return s;   // else: an exp table too large for shared memory
+        const nm_status s = nm_launch_attention_stream(ctx, d, st, out_q, q_inv_scale);
+        if (s != NM_ERR_UNSUPPORTED) {   // else: an exp table too large for shared memory
+            if (fused && out_q && s == NM_OK) *fused = true;
+            return s;
+        }
     }
     return nm_launch_attention_simt(ctx, d, st);
 }
 
-nm_status nm_layernorm_pwl(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
-                           int64_t rows, int32_t H, float eps, int32_t rsqrt_slot, nm_dtype dtype, void* stream)
+// q != nullptr: the kernel also writes the int8 codes of its (rounded) output, scale 1/q_inv_scale
+static nm_status layernorm_checked(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
+                                   int64_t rows, int32_t H, float eps, int32_t rsqrt_slot, nm_dtype dtype, void* stream,
+                                   int8_t* q, float q_inv_scale)
 {
     if (!ctx) return NM_ERR_INVALID_ARG;
     if (rows < 0 || H < 0) return NM_ERR_SHAPE;
@@ -359,7 +376,14 @@ nm_status nm_layernorm_pwl(nm_ctx* ctx, const void* x, const float* gamma, const
     if (!x || !y || !gamma || !beta) return NM_ERR_INVALID_ARG;
     if (H % 8 != 0) return NM_ERR_SHAPE;
     if (!nm_aligned16(x) || !nm_aligned16(y) || !nm_aligned16(gamma) || !nm_aligned16(beta)) return NM_ERR_ALIGNMENT;
-    return nm_launch_layernorm(ctx, x, gamma, beta, y, rows, H, eps, rsqrt_slot, NM_SLOT_NONE, dtype, (cudaStream_t)stream);
+    return nm_launch_layernorm(ctx, x, gamma, beta, y, rows, H, eps, rsqrt_slot, NM_SLOT_NONE, dtype, (cudaStream_t)stream,
+                               q, q_inv_scale);
+}
+
+nm_status nm_layernorm_pwl(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
+                           int64_t rows, int32_t H, float eps, int32_t rsqrt_slot, nm_dtype dtype, void* stream)
+{
+    return layernorm_checked(ctx, x, gamma, beta, y, rows, H, eps, rsqrt_slot, dtype, stream, nullptr, 0.f);
 }
 
 nm_status nm_layernorm_pwl_sqrt_recip(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
@@ -431,8 +455,24 @@ size_t nm_encoder_workspace_bytes(const nm_encoder_cfg* cfg)
     return lo.total;
 }
 
+// The int8 layer quantises three activations (its input, the attention output, LN1's output).  The
+// producing kernels write those int8 codes themselves where they can (LayerNorm and the streaming
+// attention kernel), so no separate pass re-reads the activation.  Within a stack the previous layer's
+// LN2 has already left the codes of this layer's input in the workspace (`in_codes_ready`), and this
+// layer's LN2 leaves those of the next (`next_a_x` > 0: the next layer's input scale).
+static nm_status encoder_layer_impl(nm_ctx* ctx, const nm_encoder_weights* w, const nm_encoder_cfg* c, const void* x,
+                                    void* y, void* workspace, size_t ws_bytes, void* stream, bool in_codes_ready,
+                                    float next_a_x);
+
 nm_status nm_encoder_layer(nm_ctx* ctx, const nm_encoder_weights* w, const nm_encoder_cfg* c, const void* x, void* y,
                            void* workspace, size_t ws_bytes, void* stream)
+{
+    return encoder_layer_impl(ctx, w, c, x, y, workspace, ws_bytes, stream, false, 0.f);
+}
+
+static nm_status encoder_layer_impl(nm_ctx* ctx, const nm_encoder_weights* w, const nm_encoder_cfg* c, const void* x,
+                                    void* y, void* workspace, size_t ws_bytes, void* stream, bool in_codes_ready,
+                                    float next_a_x)
 {
     if (!ctx || !w || !c || !x || !y) return NM_ERR_INVALID_ARG;
     EncLayout lo;
@@ -473,8 +513,10 @@ nm_status nm_encoder_layer(nm_ctx* ctx, const nm_encoder_weights* w, const nm_en
     // qkv = x Wqkv^T + bqkv
     const void* a_in = x;
     if (i8) {
-        s = nm_quantize_i8(ctx, x, act, T * H, 1.0f / w->a_x, q8, stream);
-        if (s != NM_OK) return s;
+        if (!in_codes_ready) {
+            s = nm_quantize_i8(ctx, x, act, T * H, 1.0f / w->a_x, q8, stream);
+            if (s != NM_OK) return s;
+        }
         a_in = q8;
     }
     s = linear(a_in, H, w->Wqkv, 3 * H, w->bqkv, nullptr, NM_SLOT_NONE, qkv, act, w->a_x, w->s_wqkv, 0.f);
@@ -489,28 +531,27 @@ nm_status nm_encoder_layer(nm_ctx* ctx, const nm_encoder_weights* w, const nm_en
     ad.stride_b = (int64_t)c->L * 3 * H; ad.stride_t = 3 * H;
     ad.scale = 1.0f / sqrtf((float)d);
     ad.exp_slot = c->exp_slot; ad.recip_slot = c->recip_slot; ad.out = attn; ad.algo = c->algo;
-    s = nm_attention_pwl(ctx, &ad, stream);
+    bool attn_codes = false;
+    s = attention_dispatch(ctx, &ad, stream, i8 ? q8 : nullptr, i8 ? 1.0f / w->a_attn : 0.f, &attn_codes);
     if (s != NM_OK) return s;
 
     // z = x + a Wo^T + bo ; x1 = LN1(z)
     a_in = attn;
     if (i8) {
-        s = nm_quantize_i8(ctx, attn, act, T * H, 1.0f / w->a_attn, q8, stream);
-        if (s != NM_OK) return s;
+        if (!attn_codes) {
+            s = nm_quantize_i8(ctx, attn, act, T * H, 1.0f / w->a_attn, q8, stream);
+            if (s != NM_OK) return s;
+        }
         a_in = q8;
     }
     s = linear(a_in, H, w->Wo, H, w->bo, x, NM_SLOT_NONE, z, act, w->a_attn, w->s_wo, 0.f);
     if (s != NM_OK) return s;
-    s = nm_layernorm_pwl(ctx, z, w->g1, w->be1, x1, T, H, c->eps, c->rsqrt_slot, act, stream);
+    s = layernorm_checked(ctx, z, w->g1, w->be1, x1, T, H, c->eps, c->rsqrt_slot, act, stream, i8 ? q8 : nullptr,
+                          i8 ? 1.0f / w->a_x1 : 0.f);
     if (s != NM_OK) return s;
 
     // g = PWLgelu(x1 W1^T + b1)   (int8 path: requantised in the epilogue with the scale of g)
-    a_in = x1;
-    if (i8) {
-        s = nm_quantize_i8(ctx, x1, act, T * H, 1.0f / w->a_x1, q8, stream);
-        if (s != NM_OK) return s;
-        a_in = q8;
-    }
+    a_in = i8 ? (const void*)q8 : (const void*)x1;
     if (i8) s = linear(a_in, H, w->W1, F, w->b1, nullptr, c->gelu_slot, g, NM_I8, w->a_x1, w->s_w1, 1.0f / w->a_g);
     else s = linear(a_in, H, w->W1, F, w->b1, nullptr, c->gelu_slot, g, act, 0.f, nullptr, 0.f);
     if (s != NM_OK) return s;
@@ -518,7 +559,9 @@ nm_status nm_encoder_layer(nm_ctx* ctx, const nm_encoder_weights* w, const nm_en
     // y = LN2(x1 + g W2^T + b2)
     s = linear(g, F, w->W2, H, w->b2, x1, NM_SLOT_NONE, z, act, w->a_g, w->s_w2, 0.f);
     if (s != NM_OK) return s;
-    return nm_layernorm_pwl(ctx, z, w->g2, w->be2, y, T, H, c->eps, c->rsqrt_slot, act, stream);
+    const bool chain = i8 && next_a_x > 0.f;
+    return layernorm_checked(ctx, z, w->g2, w->be2, y, T, H, c->eps, c->rsqrt_slot, act, stream, chain ? q8 : nullptr,
+                             chain ? 1.0f / next_a_x : 0.f);
 }
 
 nm_status nm_encoder_stack(nm_ctx* ctx, const nm_encoder_weights* layers, int32_t n_layers, const nm_encoder_cfg* c,
@@ -532,10 +575,14 @@ nm_status nm_encoder_stack(nm_ctx* ctx, const nm_encoder_weights* layers, int32_
     // layer outputs alternate between y and a workspace buffer so that the last one lands in y
     void* pp = (uint8_t*)workspace + lo.pingpong;
     const void* in = x;
+    bool codes_ready = false;
     for (int l = 0; l < n_layers; ++l) {
         const bool to_y = ((n_layers - 1 - l) % 2) == 0;
         void* out = to_y ? y : pp;
-        nm_status s = nm_encoder_layer(ctx, &layers[l], c, in, out, workspace, ws_bytes, stream);
+        // int8: LN2 of layer l leaves the codes of layer l+1's input in the workspace
+        const float next_a_x = (c->dtype == NM_I8 && l + 1 < n_layers) ? layers[l + 1].a_x : 0.f;
+        nm_status s = encoder_layer_impl(ctx, &layers[l], c, in, out, workspace, ws_bytes, stream, codes_ready, next_a_x);
+        codes_ready = next_a_x > 0.f;
         if (s != NM_OK) return s;
         in = out;
     }

@@ -595,7 +595,8 @@ nm_status nm_launch_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int
                               int32_t* idx_out, cudaStream_t st);
 nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
                               int64_t rows, int32_t H, float eps, int32_t slot, int32_t slot2, nm_dtype dtype,
-                              cudaStream_t st);   // slot2 != NM_SLOT_NONE: sqrt in slot, 1/x in slot2
+                              cudaStream_t st, int8_t* q = nullptr, float q_inv_scale = 0.f);
+// slot2 != NM_SLOT_NONE: sqrt in slot, 1/x in slot2; q != nullptr: also the int8 codes of the stored output
 nm_status nm_launch_wait_selftest(nm_ctx* ctx, long long limit_cycles, cudaStream_t st);
 nm_status nm_launch_quantize(nm_ctx* ctx, const void* x, nm_dtype dtype, int64_t count, float inv_scale,
                              int8_t* q, cudaStream_t st);
@@ -605,7 +606,10 @@ bool nm_linear_tc_supported(const nm_linear_desc* d);
 nm_status nm_launch_attention_simt(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
 nm_status nm_launch_attention_tc(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
 bool nm_attention_tc_supported(const nm_attn_desc* d);
-nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st);
+// out_q != nullptr: the output is written as int8 codes (of the value rounded to the storage type) to out_q
+// [B*L, heads*d] instead of d->out
+nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st, int8_t* out_q = nullptr,
+                                     float q_inv_scale = 0.f);
 bool nm_attention_stream_supported(const nm_attn_desc* d);
 nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int Nb, int H, int W, int Cin, int kh,
                            int kw, int stride, int pad, int Ho, int Wo, int Kpad, cudaStream_t st);

@@ -80,7 +80,8 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restric
                                                         const NmTable* __restrict__ tab2, const T* __restrict__ x,
                                                         const float* __restrict__ gamma,
                                                         const float* __restrict__ beta, T* __restrict__ y,
-                                                        int64_t rows, int H, float eps)
+                                                        int64_t rows, int H, float eps, int8_t* __restrict__ q,
+                                                        float q_inv_scale)
 {
     // A warp walks over rows with a grid-wide stride; the raw 16-byte vectors of its NEXT row are
     // already in flight while the current row is reduced and written, so every SM keeps several
@@ -165,6 +166,15 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restric
 #pragma unroll
                 for (int i = 0; i < N; ++i) f[it][i] = __fmaf_rn(f[it][i] * r, g[i], b[i]);
                 store16<T>(yr + v * N, f[it]);
+                if (q) {   // the int8 code of the value as stored (rounded to T first), for the next int8 GEMM
+                    int8_t code[N];
+#pragma unroll
+                    for (int i = 0; i < N; ++i)
+                        code[i] = nm_quant_i8(NmType<T>::to_f(NmType<T>::from_f(f[it][i])), q_inv_scale);
+                    int8_t* qp = q + row * H + v * N;
+                    if constexpr (N == 8) *reinterpret_cast<uint2*>(qp) = *reinterpret_cast<const uint2*>(code);
+                    else *reinterpret_cast<uint32_t*>(qp) = *reinterpret_cast<const uint32_t*>(code);
+                }
             }
         }
     }
@@ -217,7 +227,7 @@ __global__ void wait_selftest_kernel(int* status, long long limit_cycles, int* r
 
 template <typename T>
 nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const NmTable* tab2, const void* x, const float* gamma, const float* beta, void* y,
-                    int64_t rows, int H, float eps, cudaStream_t st)
+                    int64_t rows, int H, float eps, int8_t* q, float q_inv_scale, cudaStream_t st)
 {
     constexpr int N = VecOf<T>::N;
     const int nvec = H / N;
@@ -239,7 +249,8 @@ nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const NmTable* tab2, const 
     cfg.numAttrs = ctx->pdl ? 1 : 0;
     const T* xt = (const T*)x;
     T* yt = (T*)y;
-#define NM_LN_CASE(I) cudaLaunchKernelEx(&cfg, layernorm_kernel<T, I>, tab, tab2, xt, gamma, beta, yt, rows, H, eps)
+#define NM_LN_CASE(I) \
+    cudaLaunchKernelEx(&cfg, layernorm_kernel<T, I>, tab, tab2, xt, gamma, beta, yt, rows, H, eps, q, q_inv_scale)
     if (iters <= 1) NM_LN_CASE(1);
     else if (iters <= 2) NM_LN_CASE(2);
     else if (iters <= 3) NM_LN_CASE(3);
@@ -284,14 +295,14 @@ nm_status nm_launch_pwl_apply(nm_ctx* ctx, int slot, const void* x, void* y, int
 
 nm_status nm_launch_layernorm(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
                               int64_t rows, int32_t H, float eps, int32_t slot, int32_t slot2, nm_dtype dtype,
-                              cudaStream_t st)
+                              cudaStream_t st, int8_t* q, float q_inv_scale)
 {
     const NmTable* tab = ctx->d_tables + slot;
     const NmTable* tab2 = slot2 == NM_SLOT_NONE ? nullptr : ctx->d_tables + slot2;
     switch (dtype) {
-    case NM_F32: return launch_ln<float>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, st);
-    case NM_BF16: return launch_ln<__nv_bfloat16>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, st);
-    case NM_F16: return launch_ln<__half>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, st);
+    case NM_F32: return launch_ln<float>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, q, q_inv_scale, st);
+    case NM_BF16: return launch_ln<__nv_bfloat16>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, q, q_inv_scale, st);
+    case NM_F16: return launch_ln<__half>(ctx, tab, tab2, x, gamma, beta, y, rows, H, eps, q, q_inv_scale, st);
     default: return NM_ERR_UNSUPPORTED;
     }
 }
