@@ -18,51 +18,77 @@ __global__ void __launch_bounds__(256) im2col_vec_kernel(const T* __restrict__ x
                                                          int W, int Cin, int kh, int kw, int stride, int pad,
                                                          int Ho, int Wo)
 {
+    // Chunk i of A is (m, ky, kx, c8) = (output pixel, tap, 8 channels), in that order of significance.  A
+    // thread visits i, i + step, i + 2 step, ...: its coordinates are decomposed once (the only divisions)
+    // and then advanced by the decomposition of `step` with carries, so that the loop is address
+    // arithmetic, one 16-byte load and one 16-byte store.
     const int c8n = Cin >> 3;
     const int64_t chunks_per_row = (int64_t)kh * kw * c8n;
     const int64_t total = (int64_t)Nb * Ho * Wo * chunks_per_row;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += step) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    int c8, kx, ky, ox, oy, n;
+    {
         const int64_t m = i / chunks_per_row;
         const int r = (int)(i - m * chunks_per_row);
-        const int c8 = r % c8n;
-        const int kx = (r / c8n) % kw;
-        const int ky = r / (c8n * kw);
-        const int ox = (int)(m % Wo);
-        const int oy = (int)((m / Wo) % Ho);
-        const int n = (int)(m / ((int64_t)Wo * Ho));
+        c8 = r % c8n; kx = (r / c8n) % kw; ky = r / (c8n * kw);
+        ox = (int)(m % Wo); oy = (int)((m / Wo) % Ho); n = (int)(m / ((int64_t)Wo * Ho));
+    }
+    int dc8, dkx, dky, dox, doy, dn;
+    {
+        const int64_t dm = step / chunks_per_row;
+        const int dr = (int)(step - dm * chunks_per_row);
+        dc8 = dr % c8n; dkx = (dr / c8n) % kw; dky = dr / (c8n * kw);
+        dox = (int)(dm % Wo); doy = (int)((dm / Wo) % Ho); dn = (int)(dm / ((int64_t)Wo * Ho));
+    }
+    for (; i < total; i += step) {
         const int iy = oy * stride - pad + ky, ix = ox * stride - pad + kx;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (iy >= 0 && iy < H && ix >= 0 && ix < W)
             v = __ldg(reinterpret_cast<const uint4*>(x + (((int64_t)n * H + iy) * W + ix) * Cin + c8 * 8));
         *reinterpret_cast<uint4*>(A + i * 8) = v;
+        // advance by `step`: every digit gains its share plus the carry of the digit below (each at most once)
+        c8 += dc8; if (c8 >= c8n) { c8 -= c8n; ++kx; }
+        kx += dkx; if (kx >= kw) { kx -= kw; ++ky; }
+        ky += dky; if (ky >= kh) { ky -= kh; ++ox; }
+        ox += dox; if (ox >= Wo) { ox -= Wo; ++oy; }
+        oy += doy; if (oy >= Ho) { oy -= Ho; ++n; }
+        n += dn;
     }
 }
 
-// Scalar path (first layer, Cin = 3): rows padded with zeros to Kpad (a multiple of 8).
+// Path for a channel count that is not a multiple of 8 (first layer, Cin = 3): rows padded with zeros
+// to Kpad (a multiple of 8).  One thread per 16-byte chunk of A = 8 consecutive k of one output pixel;
+// k = (ky*kw + kx)*Cin + c is decomposed once per chunk and stepped with carries, the elements are
+// gathered one by one (they are adjacent in x only within a pixel) and leave as one 16-byte store.
 template <typename T>
 __global__ void __launch_bounds__(256) im2col_scalar_kernel(const T* __restrict__ x, T* __restrict__ A, int Nb, int H,
                                                             int W, int Cin, int kh, int kw, int stride, int pad,
                                                             int Ho, int Wo, int Kpad)
 {
     const int K = kh * kw * Cin;
-    const int64_t total = (int64_t)Nb * Ho * Wo * Kpad;
+    const int cpr = Kpad >> 3;   // chunks per row
+    const int64_t total = (int64_t)Nb * Ho * Wo * cpr;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += step) {
-        const int64_t m = i / Kpad;
-        const int k = (int)(i - m * Kpad);
-        T v = NmType<T>::from_f(0.f);
-        if (k < K) {
-            const int c = k % Cin;
-            const int kx = (k / Cin) % kw;
-            const int ky = k / (Cin * kw);
-            const int ox = (int)(m % Wo);
-            const int oy = (int)((m / Wo) % Ho);
-            const int n = (int)(m / ((int64_t)Wo * Ho));
-            const int iy = oy * stride - pad + ky, ix = ox * stride - pad + kx;
-            if (iy >= 0 && iy < H && ix >= 0 && ix < W) v = x[(((int64_t)n * H + iy) * W + ix) * Cin + c];
+        const int64_t m = i / cpr;
+        const int k0 = (int)(i - m * cpr) * 8;
+        const int ox = (int)(m % Wo);
+        const int oy = (int)((m / Wo) % Ho);
+        const int n = (int)(m / ((int64_t)Wo * Ho));
+        int c = k0 % Cin, kx = (k0 / Cin) % kw, ky = k0 / (Cin * kw);
+        const T* xn = x + (int64_t)n * H * W * Cin;
+        const int y0 = oy * stride - pad, x0 = ox * stride - pad;
+        T v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int iy = y0 + ky, ix = x0 + kx;
+            v[e] = NmType<T>::from_f(0.f);
+            if (k0 + e < K && iy >= 0 && iy < H && ix >= 0 && ix < W) v[e] = xn[((int64_t)iy * W + ix) * Cin + c];
+            if (++c == Cin) { c = 0; if (++kx == kw) { kx = 0; ++ky; } }
         }
-        A[i] = v;
+        *reinterpret_cast<uint4*>(A + i * 8) = *reinterpret_cast<const uint4*>(v);
     }
 }
 
@@ -176,7 +202,7 @@ nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int
         else
             im2col_vec_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)A, Nb, H, W, Cin, kh, kw, stride, pad, Ho, Wo);
     } else {
-        const int64_t total = M * Kpad;
+        const int64_t total = M * (Kpad / 8);
         if (dt == NM_F16)
             im2col_scalar_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)A, Nb, H, W, Cin, kh, kw, stride, pad, Ho, Wo, Kpad);
         else
