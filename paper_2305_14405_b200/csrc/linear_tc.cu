@@ -127,7 +127,10 @@ template <> __device__ __forceinline__ void add_res32<float>(const uint32_t* w, 
 }
 template <> __device__ __forceinline__ void add_res32<int8_t>(const uint32_t*, float*) {}
 
-template <typename InT, typename OutT, bool TWO>
+// NV < 4 (16-bit outputs, no residual, one tile across N): only the first NV groups of 64 columns of the
+// tile exist; the epilogue takes just those (a narrow layer under the 256-wide tile is epilogue-bound
+// otherwise: the accumulator columns beyond N hold products with zero-filled weight rows).
+template <typename InT, typename OutT, bool TWO, int NV = 4>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                  const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmR, const TcArgs a)
@@ -377,9 +380,23 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool row_ok = row < a.M;
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2));
             uint32_t r[2][32];
-            nm_tmem_ld32_async(t_addr, r[0]);
+            int nchv = NCH;   // chunks of 32 columns this warp takes from the tile
+            if constexpr (NV < 4) {
+                const int ngv = half == 0 ? (NV < 2 ? NV : 2) : (NV > 2 ? NV - 2 : 0);
+                nchv = ngv * GC;
+                if (nchv == 0) {   // nothing to read: hand the accumulator back at once
+                    nm_tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) nm_mbar_arrive(&bar_acc_empty[buf]);
+                    __syncwarp();
+                }
+            }
+            if (nchv > 0) nm_tmem_ld32_async(t_addr, r[0]);
 #pragma unroll
             for (int g = 0; g < NG; ++g) {
+                if constexpr (NV < 4) {
+                    if (g * GC >= nchv) continue;
+                }
                 uint32_t packed[32];
                 uint32_t rsv[32];
                 if (has_res) {
@@ -415,7 +432,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const int c = g * GC + cc;
                     const int cur = c & 1;
                     nm_tmem_ld_wait32(r[cur]);
-                    if (c + 1 < NCH) {
+                    if (c + 1 < (NV < 4 ? nchv : NCH)) {
                         nm_tmem_ld32_async(t_addr + (uint32_t)((c + 1) * 32), r[cur ^ 1]);
                     } else {
                         // this warp's share of the accumulator is in registers: hand the buffer back
@@ -536,7 +553,7 @@ nm_status make_tmap(nm_ctx* ctx, CUtensorMap* m, const void* base, nm_dtype dt, 
     return r == CUDA_SUCCESS ? NM_OK : NM_ERR_CUDA;
 }
 
-template <typename InT, typename OutT, bool TWO>
+template <typename InT, typename OutT, bool TWO, int NV = 4>
 nm_status launch(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
 {
     constexpr int B_ROWS = TWO ? BN / 2 : BN;
@@ -580,7 +597,7 @@ nm_status launch(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
     else tmR = tmO;
     if (s != NM_OK) return s;
 
-    auto kern = linear_tc_kernel<InT, OutT, TWO>;
+    auto kern = linear_tc_kernel<InT, OutT, TWO, NV>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return NM_ERR_CUDA;
     cudaLaunchConfig_t cfg;
@@ -627,6 +644,10 @@ nm_status launch_sel(nm_ctx* ctx, const nm_linear_desc* d, cudaStream_t st)
 {
     // algo 3 forces the one-CTA tile; otherwise problems with at least one 256 x 256 tile use CTA pairs
     if (d->algo != 3 && d->M >= 256 && d->N >= 256) return launch<InT, OutT, true>(ctx, d, st);
+    if constexpr (sizeof(OutT) == 2) {   // narrow layers: the epilogue takes the existing column groups only
+        if (!d->residual && d->N <= 64) return launch<InT, OutT, false, 1>(ctx, d, st);
+        if (!d->residual && d->N <= 128) return launch<InT, OutT, false, 2>(ctx, d, st);
+    }
     return launch<InT, OutT, false>(ctx, d, st);
 }
 
