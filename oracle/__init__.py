@@ -348,6 +348,29 @@ def maxpool_nhwc(x, ksz, stride, pad):
     return out
 
 
+def maxpool_nhwc_relu(x, ksz, stride, pad, t_relu: Table):
+    """Max pooling with the maximum itself written as the paper's operator form (Section 3: a network of
+    linear operators and PWL nonlinearities): max(a, b) = b + PWLrelu(a - b), folded over the window in
+    raster order; the first cell inside the image starts the fold, padding cells are skipped."""
+    x = _f64(x)
+    Nb, Hin, Win, Cc = x.shape
+    Ho = (Hin + 2 * pad - ksz) // stride + 1
+    Wo = (Win + 2 * pad - ksz) // stride + 1
+    out = np.empty((Nb, Ho, Wo, Cc))
+    for oy in range(Ho):
+        for ox in range(Wo):
+            m = None
+            for ky in range(ksz):
+                for kx in range(ksz):
+                    iy, ix = oy * stride - pad + ky, ox * stride - pad + kx
+                    if iy < 0 or iy >= Hin or ix < 0 or ix >= Win:
+                        continue
+                    v = x[:, iy, ix, :]
+                    m = v.copy() if m is None else m + pwl_eval(t_relu, v - m)[0]
+            out[:, oy, ox, :] = m
+    return out
+
+
 def avgpool_nhwc(x):
     x = _f64(x)
     Nb, Hin, Win, Cc = x.shape

@@ -542,6 +542,28 @@ def test_int8_encoder_layer_against_library_routines():
     assert (err > 1e-9).mean() < 0.02 and np.median(err) < 1e-12
 
 
+def test_maxpool_relu_form_is_the_library_max_pool():
+    """max(a, b) = b + ReLU(a - b): with the 2-segment ReLU table (exact everywhere) and fp16-representable
+    inputs every difference and sum is exact in fp64, so the fold reproduces torch's max pooling exactly,
+    padding and stride included."""
+    rng = np.random.default_rng(21)
+    x = nm_inputs.round_to(rng.standard_normal((2, 9, 11, 5)).astype(np.float32) * 3, "f16").astype(np.float64)
+    relu = Table.secant(oracle.RELU, 2, -8.0, 8.0)
+    for ks, st, pad in ((3, 2, 1), (2, 2, 0), (3, 1, 1)):
+        got = oracle.maxpool_nhwc_relu(x, ks, st, pad, relu)
+        ref = torch.nn.functional.max_pool2d(torch.from_numpy(x).permute(0, 3, 1, 2), ks, st, pad).permute(0, 2, 3, 1)
+        assert np.array_equal(got, ref.numpy())
+        assert np.array_equal(got, oracle.maxpool_nhwc(x, ks, st, pad))
+
+
+def test_maxpool_relu_form_uses_the_table():
+    """With a table that is not ReLU the fold is no longer a maximum: b + t(a - b) on a 1 x 2 window."""
+    half = Table(2, -8.0, 8.0, np.array([0.0, 0.5], np.float32), np.array([0.0, 0.0], np.float32))   # 0.5 * ReLU
+    y = oracle.maxpool_nhwc_relu(np.array([[[[1.0], [3.0]], [[0.0], [0.0]]]]), 2, 1, 0, half)
+    # fold order: (0,0)=1 -> (0,1)=3: 1 + 0.5*2 = 2 -> (1,0)=0: 2 + 0 -> (1,1)=0: 2
+    assert y.shape == (1, 1, 1, 1) and y[0, 0, 0, 0] == 2.0
+
+
 def test_resnet50_composition_against_torch():
     """The oracle's ResNet-50-shaped network (a composition of its own conv / pool / linear routines)
     against torch.nn.functional in fp64 on a reduced image: pins the block wiring (projection shortcut
