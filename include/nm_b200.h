@@ -305,6 +305,14 @@ nm_status nm_maxpool2d(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int3
 nm_status nm_avgpool_global(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,
                             int32_t C, void* stream);
 
+/* The same max pooling with the maximum evaluated in that operator form (Section 3: every
+ * operator is linear or a PWL table): over the window cells inside the image, in raster order,
+ *     m = first cell;  m = m + PWL_relu(cell - m) for every further cell,
+ * with the table in relu_slot (fp32 arithmetic).  With the 2-segment ReLU table the result equals
+ * nm_maxpool2d's.  Arguments and errors as nm_maxpool2d; NM_ERR_NO_TABLE if the slot is empty. */
+nm_status nm_maxpool2d_pwl(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,
+                           int32_t C, int32_t ks, int32_t stride, int32_t pad, int32_t relu_slot, void* stream);
+
 /* ResNet-50-shaped CNN computed entirely with GEMMs and PWL tables (Section 5 evaluates ResNet):
  * 7x7/2 convolution, 3x3/2 max-pool, 16 bottleneck blocks (1x1 -> 3x3 -> 1x1, widths 64/128/256/512
  * x4, the stride in the 3x3 convolution, 1x1 projection shortcut in the first block of a stage,

@@ -28,7 +28,7 @@ EXPORTS = [
     "nm_pwl_table_build", "nm_pwl_table_load", "nm_pwl_apply", "nm_linear_pwl", "nm_attention_pwl",
     "nm_layernorm_pwl", "nm_layernorm_pwl_sqrt_recip", "nm_quantize_i8", "nm_encoder_workspace_bytes", "nm_encoder_layer", "nm_encoder_stack",
     "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
-    "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
+    "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_maxpool2d_pwl", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
     "nm_resnet50_forward", "nm_resnet50_forward_host", "nm_pwl_table_build_elastic",
     "nm_selftest_bounded_wait",
 ]
@@ -139,6 +139,7 @@ def load():
     lib.nm_conv2d_workspace_bytes.argtypes = [C.POINTER(ConvDesc)]
     lib.nm_conv2d_pwl.argtypes = [C.c_void_p, C.POINTER(ConvDesc), C.c_void_p, C.c_size_t, C.c_void_p]
     lib.nm_maxpool2d.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_int32] * 7 + [C.c_void_p]
+    lib.nm_maxpool2d_pwl.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_int32] * 8 + [C.c_void_p]
     lib.nm_avgpool_global.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_int32] * 4 + [C.c_void_p]
     lib.nm_resnet50_workspace_bytes.restype = C.c_size_t
     lib.nm_resnet50_workspace_bytes.argtypes = [C.POINTER(Resnet50Cfg)]
@@ -362,6 +363,11 @@ class Context:
         N, H, W, Cc = x.shape
         _check(self._lib.nm_maxpool2d(self._h, _ptr(x), _ptr(y), dtype_of(x), N, H, W, Cc, ks, stride, pad,
                                       _stream(stream)), "nm_maxpool2d")
+
+    def maxpool2d_pwl(self, x, y, ks, stride, pad, relu_slot=SLOT_RELU, stream=None):
+        N, H, W, Cc = x.shape
+        _check(self._lib.nm_maxpool2d_pwl(self._h, _ptr(x), _ptr(y), dtype_of(x), N, H, W, Cc, ks, stride, pad,
+                                          relu_slot, _stream(stream)), "nm_maxpool2d_pwl")
 
     def avgpool_global(self, x, y, stream=None):
         N, H, W, Cc = x.shape

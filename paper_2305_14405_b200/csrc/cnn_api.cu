@@ -107,6 +107,21 @@ nm_status nm_maxpool2d(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int3
     return nm_launch_maxpool(ctx, x, y, dtype, N, H, W, C, ks, stride, pad, Ho, Wo, (cudaStream_t)stream);
 }
 
+nm_status nm_maxpool2d_pwl(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,
+                           int32_t C, int32_t ks, int32_t stride, int32_t pad, int32_t relu_slot, void* stream)
+{
+    if (!ctx || !x || !y) return NM_ERR_INVALID_ARG;
+    if (relu_slot < 0 || relu_slot >= NM_NUM_SLOTS) return NM_ERR_INVALID_ARG;
+    if (!ctx->h_tables[relu_slot].loaded) return NM_ERR_NO_TABLE;
+    if (dtype != NM_F16 && dtype != NM_BF16) return NM_ERR_UNSUPPORTED;
+    if (N < 1 || H < 1 || W < 1 || C < 8 || C % 8 != 0 || ks < 1 || stride < 1 || pad < 0 || pad >= ks ||
+        H + 2 * pad < ks || W + 2 * pad < ks)
+        return NM_ERR_SHAPE;
+    if (!nm_aligned16(x) || !nm_aligned16(y)) return NM_ERR_ALIGNMENT;
+    const int Ho = (H + 2 * pad - ks) / stride + 1, Wo = (W + 2 * pad - ks) / stride + 1;
+    return nm_launch_maxpool(ctx, x, y, dtype, N, H, W, C, ks, stride, pad, Ho, Wo, (cudaStream_t)stream, relu_slot);
+}
+
 nm_status nm_avgpool_global(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,
                             int32_t C, void* stream)
 {

@@ -110,11 +110,15 @@ template <typename T> struct Vec2;
 template <> struct Vec2<__half> { using type = __half2; static __device__ __forceinline__ __half2 make(float a, float b) { return __floats2half2_rn(a, b); } };
 template <> struct Vec2<__nv_bfloat16> { using type = __nv_bfloat162; static __device__ __forceinline__ __nv_bfloat162 make(float a, float b) { return __floats2bfloat162_rn(a, b); } };
 
-// window maximum, padding cells ignored; 8 channels per thread
+// window maximum, padding cells ignored; 8 channels per thread.  With a table (`relu`), the maximum is
+// taken in its operator form max(a, b) = b + PWLrelu(a - b), folded over the window in raster order.
 template <typename T>
 __global__ void __launch_bounds__(256) maxpool_kernel(const T* __restrict__ x, T* __restrict__ y, int Nb, int H, int W,
-                                                      int C, int ks, int stride, int pad, int Ho, int Wo)
+                                                      int C, int ks, int stride, int pad, int Ho, int Wo,
+                                                      const NmTable* __restrict__ relu)
 {
+    float inv_h = 0.f, off = 0.f, nm1 = 0.f;
+    if (relu) { inv_h = relu->inv_h; off = relu->off; nm1 = (float)(relu->n - 1); }
     using V2 = typename Vec2<T>::type;
     const int c8n = C >> 3;
     const int64_t total = (int64_t)Nb * Ho * Wo * c8n;
@@ -125,6 +129,7 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const T* __restrict__ x, T
         float best[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) best[j] = -INFINITY;
+        bool first = true;
         for (int ky = 0; ky < ks; ++ky) {
             const int iy = oy * stride - pad + ky;
             if (iy < 0 || iy >= H) continue;
@@ -136,9 +141,23 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const T* __restrict__ x, T
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float2 f = unpack2(h[j]);
-                    best[2 * j] = fmaxf(best[2 * j], f.x);
-                    best[2 * j + 1] = fmaxf(best[2 * j + 1], f.y);
+                    if (relu && !first) {
+                        const float v[2] = {f.x, f.y};
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float dlt = v[e] - best[2 * j + e];
+                            const float2 kb = relu->kb[nm_pwl_index(dlt, inv_h, off, nm1)];
+                            best[2 * j + e] += __fmaf_rn(kb.x, dlt, kb.y);
+                        }
+                    } else if (relu) {
+                        best[2 * j] = f.x;
+                        best[2 * j + 1] = f.y;
+                    } else {
+                        best[2 * j] = fmaxf(best[2 * j], f.x);
+                        best[2 * j + 1] = fmaxf(best[2 * j + 1], f.y);
+                    }
                 }
+                first = false;
             }
         }
         uint4 out;
@@ -222,14 +241,15 @@ nm_status nm_launch_pad_rows(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, 
 }
 
 nm_status nm_launch_maxpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int H, int W, int C, int ks,
-                            int stride, int pad, int Ho, int Wo, cudaStream_t st)
+                            int stride, int pad, int Ho, int Wo, cudaStream_t st, int relu_slot)
 {
+    const NmTable* relu = relu_slot == NM_SLOT_NONE ? nullptr : ctx->d_tables + relu_slot;
     const int64_t total = (int64_t)Nb * Ho * Wo * (C / 8);
     NmLaunchScope scope(ctx, NM_KERNEL_POOL, ((double)Nb * H * W * C + (double)Nb * Ho * Wo * C) * nm_dtype_size(dt), st);
     if (dt == NM_F16)
-        maxpool_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo);
+        maxpool_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo, relu);
     else
-        maxpool_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo);
+        maxpool_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo, relu);
     return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
 }
 

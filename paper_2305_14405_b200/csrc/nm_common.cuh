@@ -616,5 +616,5 @@ nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int
 nm_status nm_launch_pad_rows(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, int rows, int K, int Kpad,
                              cudaStream_t st);
 nm_status nm_launch_maxpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int H, int W, int C, int ks,
-                            int stride, int pad, int Ho, int Wo, cudaStream_t st);
+                            int stride, int pad, int Ho, int Wo, cudaStream_t st, int relu_slot = NM_SLOT_NONE);
 nm_status nm_launch_avgpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int HW, int C, cudaStream_t st);

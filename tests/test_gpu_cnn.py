@@ -74,6 +74,28 @@ def test_pools_parity(nm, ctx):
     assert ei.value.code == 2
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("ks,stride,pad", [(3, 2, 1), (2, 2, 0), (3, 1, 1)])
+def test_maxpool_relu_form(nm, ctx, dtype, ks, stride, pad):
+    """max(a, b) = b + PWL_relu(a - b) folded over the window: equals the oracle's fold (and, with the
+    2-segment ReLU table, the plain maximum) exactly once rounded to the storage type."""
+    rng = np.random.default_rng(31 + ks)
+    x = nm_inputs.round_to(3 * rng.standard_normal((2, 21, 19, 32)).astype(np.float32), dtype)
+    k, b = ctx.load_function_table(nm.SLOT_RELU, nm.FUNC_RELU, 2, -8.0, 8.0)
+    relu = oracle.Table.secant(oracle.RELU, 2, -8.0, 8.0)
+    assert np.array_equal(np.asarray(k, np.float32), relu.k) and np.array_equal(np.asarray(b, np.float32), relu.b)
+    ref = oracle.maxpool_nhwc_relu(x, ks, stride, pad, relu)
+    td = nm_inputs.torch_dtype(dtype)
+    xd = torch.from_numpy(x).cuda().to(td)
+    y = torch.empty(ref.shape, dtype=td, device="cuda")
+    ctx.maxpool2d_pwl(xd, y, ks, stride, pad, nm.SLOT_RELU)
+    assert np.array_equal(to_np(y), ref)
+    assert np.array_equal(to_np(y), oracle.maxpool_nhwc(x, ks, stride, pad))
+    with pytest.raises(nm.NmError) as ei:
+        ctx.maxpool2d_pwl(xd, y, ks, stride, pad, 13)      # a slot that was never loaded
+    assert ei.value.code == 4
+
+
 @pytest.mark.parametrize("random_bn", [False, True])
 def test_resnet50_two_images(nm, ctx, random_bn):
     """The whole ResNet-50-shaped network (53 convolutions, pools, classifier) on two 224x224 images,

@@ -61,6 +61,7 @@ def test_calls_reject_null_context(lib):
     assert lib.nm_attention_pwl(None, None, None) == 1
     assert lib.nm_layernorm_pwl(None, None, None, None, None, 0, 0, 0.0, 0, 0, None) == 1
     assert lib.nm_layernorm_pwl_sqrt_recip(None, None, None, None, None, 0, 0, 0.0, 0, 0, 0, None) == 1
+    assert lib.nm_maxpool2d_pwl(None, None, None, 0, 0, 0, 0, 0, 0, 0, 0, 0, None) == 1
     assert lib.nm_ctx_destroy(None) == 1
     cfg = nm.Context.encoder_cfg(2, 16, 64, 4, 128, nm.BF16)
     assert lib.nm_encoder_workspace_bytes(C.byref(cfg)) > 0
