@@ -1,4 +1,4 @@
-// Fused attention with PWL softmax, streaming variant: two CTAs per SM.
+// Fused attention with PWL softmax, streaming variant: several CTAs per SM.
 //
 // Same function as attention_tc.cu (Section 3.1: attention is a linear operator; Section 3.2.2:
 // exp and 1/x as PWL tables), per query row
@@ -8,23 +8,25 @@
 // running-maximum rescaling).  Instead of keeping the whole 128 x L score block in tensor memory,
 // this kernel computes Q K^T TWICE: a first sweep over the keys only for the row maximum, a second
 // sweep for the exponentials.  The tensor pipe is idle most of the time in this ALU-bound kernel, so
-// the second Q K^T is free, and the footprint drops to 256 tensor-memory columns and ~105 KB of
-// shared memory: two CTAs fit on an SM and one CTA's loads, MMAs and barriers overlap the other's
-// arithmetic.  Any L that is a multiple of 128 is supported.
+// the second Q K^T is free, and the footprint drops to 128 tensor-memory columns and ~50 KB of
+// shared memory per softmax group (plus Q and the table): two or three CTAs fit on an SM and one
+// CTA's loads, MMAs and hand-offs overlap the others' arithmetic.  Any L that is a multiple of 128.
 //
-// The keys are split between two groups of four softmax warps, which form independent pipelines:
-// group g owns 128 tensor-memory columns [S_g | O_g], two K stages, a V stage and a P tile.  In
-// sweep 1 it takes the 128-key chunks g, g+2, ... (scores over all 128 columns, K staged in its two
-// K stages and, alternately, in its P tile); in sweep 2 the 64-key chunks g, g+2, ... (scores in
-// S_g, accumulator O_g; the two accumulators are summed in the epilogue).
+// A group is one control warp and four softmax warps, an independent pipeline that owns 128
+// tensor-memory columns [S_g | O_g], two K stages, a V stage and a P tile.  A CTA has NG = 1 or 2
+// groups (template parameter); with two, the groups split the keys: in sweep 1 group g takes the
+// 128-key chunks g, g+NG, ... (scores over all 128 columns, K staged in its two K stages and,
+// alternately, in its P tile); in sweep 2 the 64-key chunks g, g+NG, ... (scores in S_g, accumulator
+// O_g); row maxima and sums are exchanged through shared memory and the accumulators summed in the
+// epilogue.
 //
-//   warps 0-1   control warp of group 0 / 1: TMA loads (Q; the group's K chunks through two stages,
-//               its V chunks through one) and the tcgen05.mma for S_g = Q K_c^T and O_g += P_c V_c
-//               (V as an MN-major operand).  It sleeps in a named barrier (bar.sync) that the
-//               group's softmax warps signal with bar.arrive, so hand-offs cost no polling.
-//   warps 2-9   softmax, one per tensor-memory lane quarter and group: tcgen05.ld, row maximum
-//               (sweep 1); PWL exp, row sum, bf16 P tile in the swizzled K-major layout (sweep 2);
-//               PWL reciprocal, scaling, store.
+//   warps 0..NG-1     control warp of group g: TMA loads (the group's K chunks through two stages, its V
+//                     chunks through one) and the tcgen05.mma for S_g = Q K_c^T and O_g += P_c V_c (V as
+//                     an MN-major operand).  It sleeps in a named barrier (bar.sync) that the group's
+//                     softmax warps signal with bar.arrive, so hand-offs cost no polling.
+//   warps NG..5NG-1   softmax, one per tensor-memory lane quarter and group: tcgen05.ld, row maximum
+//                     (sweep 1); PWL exp, row sum, bf16 P tile in the swizzled K-major layout (sweep 2);
+//                     PWL reciprocal, scaling, store (optionally as int8 codes for the int8 encoder).
 #include <string.h>
 
 #include "nm_common.cuh"

@@ -344,7 +344,7 @@ static nm_status attention_dispatch(nm_ctx* ctx, const nm_attn_desc* d, void* st
     if (d->stride_t < (int64_t)d->heads * d->d || d->stride_b < (int64_t)d->L * d->stride_t) return NM_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (d->algo == 1) return nm_launch_attention_simt(ctx, d, st);
-    // tensor-core kernels: the streaming one (two CTAs per SM, any L that is a multiple of 128) is the
+    // tensor-core kernels: the streaming one (several CTAs per SM, any L that is a multiple of 128) is the
     // default; algo 3 selects the one that keeps the whole score block in tensor memory (L <= 512)
     if (d->algo == 3) return nm_attention_tc_supported(d) ? nm_launch_attention_tc(ctx, d, st) : NM_ERR_UNSUPPORTED;
     if (d->algo == 0 && ctx->attn_resident && nm_attention_tc_supported(d)) {
