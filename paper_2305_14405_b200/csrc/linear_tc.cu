@@ -259,8 +259,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t acc_phase = 0;
             bool ok = true;
             for (int tile = tile_first; ok && tile < a.num_tiles; tile += tile_step) {
-                if (!__all_sync(0xffffffffu, TWO ? nm_mbar_wait_cluster(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status)
-                                                 : nm_mbar_wait(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status))) { ok = false; break; }
+                // CTA-scope acquire also where the peer CTA's epilogue warps arrive: what the hand-back orders are
+                // tcgen05 operations, ordered by tcgen05.fence (a cluster-scope acquire costs ~400 cycles per tile)
+                if (!__all_sync(0xffffffffu, nm_mbar_wait(&bar_acc_empty[buf], acc_phase ^ 1u, abortp, a.status))) { ok = false; break; }
                 nm_tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
