@@ -27,9 +27,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, mean over the four
-# GEMM shapes of a layer, from the ncu capture summarised in profiles/encoder_c3_launches_and_kernels.md
-NCU_GEMM_DRAM_BYTES_PER_LAUNCH = {"c3_bert_base_12l_bf16": 82.6e6}
+NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16 / fp16 tensor peak of the part, for context
+NOMINAL_HBM_GBS = 8000.0
+REPEATS = 5                       # the K-step timed region is repeated; value = median over the repeats
 
 
 def parse_args():
@@ -47,6 +47,9 @@ def parse_args():
     p.add_argument("--hidden", type=int, default=0, help="encoder workloads: override H (heads = H/64, F = 4H)")
     p.add_argument("--layers", type=int, default=0, help="encoder workloads: override the number of layers")
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-rows-leg", action="store_true",
+                   help="encoder workloads: skip the row-kernel bandwidth leg on a tensor beyond L2")
+    p.add_argument("--repeats", type=int, default=REPEATS, help="how many times the K-step timed region is run")
     p.add_argument("--algo", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     return p.parse_args()
 
@@ -68,6 +71,7 @@ class ClockSampler(threading.Thread):
         self.index = index
         self.samples = []
         self.reasons = set()
+        self.reason_samples = {}
         self.max_mhz = None
         self.power = []
         self._stop_evt = threading.Event()
@@ -94,7 +98,8 @@ class ClockSampler(threading.Thread):
                 for bit, name in names.items():
                     if mask & bit:
                         self.reasons.add(name)
-                time.sleep(0.02)
+                        self.reason_samples[name] = self.reason_samples.get(name, 0) + 1
+                time.sleep(0.005)
         except Exception as e:  # NVML missing: report that rather than invent clocks
             self.error = repr(e)
 
@@ -107,7 +112,7 @@ class ClockSampler(threading.Thread):
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "error": self.error}
         s = sorted(self.samples)
         out = {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-               "samples": len(s)}
+               "samples": len(s), "sm_mhz_min": s[0], "reason_samples": dict(self.reason_samples)}
         if self.power:
             out["power_w_max"] = round(max(self.power), 1)
         return out
@@ -482,6 +487,58 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+def pick_peak(peaks, clocks, scale=1.0):
+    """Which measured bf16 peak a tensor-bound kernel of this run is held against: the burst figure when the
+    run kept its clocks (median SM clock within 5 % of the maximum and no power-cap sample while the kernels
+    were timed), the sustained figure otherwise.  Returns (peak, name)."""
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    held = bool(mhz and mx and mhz >= 0.95 * mx and "sw_power_cap" not in clocks.get("reasons", []))
+    name = "bf16_tflops" if held else "bf16_tflops_sustained"
+    return scale * peaks[name], ("burst" if held else "sustained")
+
+
+def fractions(achieved, peaks, scale=1.0):
+    return {"frac_burst": achieved / (scale * peaks["bf16_tflops"]),
+            "frac_sustained": achieved / (scale * peaks["bf16_tflops_sustained"]),
+            "frac_nominal": achieved / (scale * NOMINAL_BF16_TFLOPS)}
+
+
+def rows_leg(ctx, nm, dev, peaks, peak_kind, hidden=768, rows=1 << 19, iters=20):
+    """The HBM-bound row kernels (PWL LayerNorm, element-wise PWL GELU) on a tensor several times the L2
+    (805 MB per tensor at the default size), timed per launch by the library's own events: algorithmic
+    bytes (one read and one write per element) / event time, against the measured HBM copy."""
+    import torch
+    import nm_inputs
+    ctx.load_function_table(nm.SLOT_USER0 + 2, nm.FUNC_RSQRT, 64, 0.05, 8.0)
+    ctx.load_function_table(nm.SLOT_USER0 + 3, nm.FUNC_GELU, 64, -8.0, 8.0)
+    xb = nm_inputs.matrix((1 << 14, hidden), 1234, "bf16", 1.0)
+    x = torch.from_numpy(xb).to(dev).bfloat16().repeat(rows // (1 << 14), 1).contiguous()
+    g = torch.from_numpy(nm_inputs.matrix((hidden,), 1235, "f32", 0.1) + 1.0).to(dev)
+    b = torch.from_numpy(nm_inputs.matrix((hidden,), 1236, "f32", 0.1)).to(dev)
+    y = torch.empty_like(x)
+    z = torch.empty_like(x)
+    for _ in range(3):
+        ctx.layernorm_pwl(x, g, b, y, rsqrt_slot=nm.SLOT_USER0 + 2)
+        ctx.pwl_apply(nm.SLOT_USER0 + 3, y, z)
+    torch.cuda.synchronize()
+    ctx.profile_enable(True)
+    for _ in range(iters):
+        ctx.layernorm_pwl(x, g, b, y, rsqrt_slot=nm.SLOT_USER0 + 2)
+        ctx.pwl_apply(nm.SLOT_USER0 + 3, y, z)
+    torch.cuda.synchronize()
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    out = {"tensor": "[%d, %d] bf16, %.0f MB per tensor (L2 is 126 MB)" % (rows, hidden, rows * hidden * 2 / 1e6)}
+    for kind in ("layernorm", "pwl_apply"):
+        n_k, ms_k, work_k = prof[kind]
+        gbs = work_k / (ms_k * 1e-3) / 1e9 if ms_k > 0 else 0.0
+        out[kind] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": gbs / peaks["hbm_gbs"], "frac_nominal": gbs / NOMINAL_HBM_GBS, "launches": n_k,
+                     "avg_launch_us": ms_k / max(n_k, 1) * 1e3, "peak_source": "%s (HBM copy)" % peak_kind}
+    del x, y, z
+    return out
+
+
 def main():
     args = parse_args()
     wl = make_workload(args)
@@ -518,32 +575,42 @@ def main():
         wl.step()
     ctx.check_device_status()
 
-    # ---- timed region: K steps, CUDA events on the launching stream ------------------------
+    # ---- timed region: K steps between two CUDA events on the launching stream, barrier and synchronize
+    # on both sides, max over ranks; run `repeats` times, the reported time is the median ----------------
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
     time.sleep(0.05)
-    ev0 = torch.cuda.Event(enable_timing=True)
-    ev1 = torch.cuda.Event(enable_timing=True)
-    ctx.launch_count(reset=True)
-    barrier()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        wl.step()
-    ev1.record(stream)
-    barrier()
-    ms_step = max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
-    launches = ctx.launch_count()
+    reps = []
+    launches = 0
+    for _ in range(max(1, args.repeats)):
+        ev0 = torch.cuda.Event(enable_timing=True)
+        ev1 = torch.cuda.Event(enable_timing=True)
+        ctx.launch_count(reset=True)
+        barrier()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            wl.step()
+        ev1.record(stream)
+        barrier()
+        reps.append(max_over_ranks(ev0.elapsed_time(ev1)) / args.steps)
+        launches = ctx.launch_count()
     sampler.stop()
     ctx.check_device_status()
+    srt = sorted(reps)
+    ms_step = srt[len(srt) // 2]
     value = world * wl.units_per_step / (ms_step * 1e-3)
 
-    # ---- per-kernel pass: the same steps with every launch bracketed by events -------------
+    # ---- per-kernel pass: the same steps with every launch bracketed by events, clocks sampled ---------
     per_step = max(1, launches // max(args.steps, 1))
     prof_steps = min(args.steps, max(1, 8000 // per_step))
+    prof_sampler = ClockSampler(physical_gpu_index(local))
+    prof_sampler.start()
+    time.sleep(0.02)
     ctx.profile_enable(True)
     for _ in range(prof_steps):
         wl.step()
     torch.cuda.synchronize()
+    prof_sampler.stop()
     prof = ctx.profile_read()
     ctx.profile_enable(False)
 
@@ -562,6 +629,8 @@ def main():
 
     if rank == 0:
         peaks, peak_kind = load_peaks()
+        clocks = sampler.summary()
+        prof_clocks = prof_sampler.summary()
         total_ms = sum(v[1] for v in prof.values()) or 1.0
         kernels = {k: {"launches_per_step": v[0] / prof_steps, "ms_per_step": v[1] / prof_steps,
                        "share": v[1] / total_ms} for k, v in prof.items() if v[0]}
@@ -569,20 +638,28 @@ def main():
         n_l, ms_l, work_l = prof[gemm_kind]
         achieved = work_l / (ms_l * 1e-3) / 1e12 if ms_l > 0 else 0.0
         # int8: the measured bf16 peak times the nominal 2:1 int8:bf16 ratio; fp32 runs on CUDA cores
-        peak = {"i8": 2.0, "f32": 0.5}.get(wl.dtype, 1.0) * peaks["bf16_tflops_sustained"]
-        cfg_name = wl.config(world)["workload"]
+        scale = {"i8": 2.0, "f32": 0.5}.get(wl.dtype, 1.0)
+        peak, which = pick_peak(peaks, prof_clocks, scale)
         roofline = {"bound": "tensor", "kernel": gemm_kind, "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak,
-                    "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg_name),
-                    "peak_source": "%s (bf16 sustained: kernel timed inside a long step)" % peak_kind,
-                    "avg_launch_us": ms_l / max(n_l, 1) * 1e3, "share_of_step": ms_l / total_ms}
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "peak_source": "%s bf16 %s x %.1f: SM clock median %s of %s MHz, reasons %s during the per-kernel pass"
+                                   % (peak_kind, which, scale, prof_clocks.get("sm_mhz"), prof_clocks.get("sm_max_mhz"),
+                                      prof_clocks.get("reasons")),
+                    "avg_launch_us": ms_l / max(n_l, 1) * 1e3, "share_of_step": ms_l / total_ms,
+                    "work_per_step": work_l / prof_steps, "ms_per_step": ms_l / prof_steps}
+        roofline.update(fractions(achieved, peaks, scale))
+        whole = wl.flops_per_step() / (ms_step * 1e-3) / 1e12
+        wpeak, wwhich = pick_peak(peaks, clocks, scale)
+        whole_step = {"tflops": whole, "peak": wpeak, "frac": whole / wpeak, "peak_source": "%s bf16 %s x %.1f" % (peak_kind, wwhich, scale)}
+        whole_step.update(fractions(whole, peaks, scale))
         extra = {}
         for kind in ("layernorm", "quantize", "im2col", "pool"):
             n_k, ms_k, work_k = prof[kind]
             if n_k:
                 gbs = work_k / (ms_k * 1e-3) / 1e9
                 extra[kind] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": gbs / peaks["hbm_gbs"], "note": "algorithmic bytes per launch / event time"}
+                               "frac": gbs / peaks["hbm_gbs"],
+                               "note": "in the step (tensors partly L2-resident): algorithmic bytes per launch / event time"}
         for kind in ("attention_tc", "attention_simt"):
             n_a, ms_a, work_a = prof[kind]
             if n_a:
@@ -594,15 +671,20 @@ def main():
             "metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config(world),
-            "clocks": sampler.summary(),
+            "repeats": {"n": len(reps), "ms_per_step": [round(r, 5) for r in reps], "min": srt[0], "max": srt[-1],
+                        "spread": (srt[-1] - srt[0]) / ms_step, "value_is": "median"},
+            "clocks": clocks,
             "e2e": {"value": world * getattr(wl, "e2e_units", wl.units_per_step) / (e2e_ms * 1e-3), "unit": wl.unit,
                     "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": e2e_ms},
             "gpu_launches": launches,
             "roofline": roofline,
             "roofline_other": extra,
             "kernels": kernels,
-            "whole_step_tflops": wl.flops_per_step() / (ms_step * 1e-3) / 1e12,
+            "whole_step": whole_step,
+            "whole_step_tflops": whole,
         }
+        if isinstance(wl, EncoderWorkload) and not args.no_rows_leg and world == 1:
+            line["roofline_rows"] = rows_leg(ctx, nm, dev, peaks, peak_kind)
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = wl.cpu_baseline()
         print(json.dumps(line))

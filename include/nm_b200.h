@@ -18,7 +18,9 @@
  *    stream).  Work is enqueued and the call returns without waiting unless
  *    stated otherwise.
  *  - Per-call scratch comes from the caller's workspace (nm_*_workspace_bytes).
- *    The library allocates device memory only in nm_ctx_create.
+ *    The library allocates device memory only in nm_ctx_create; while per-kernel timing
+ *    (nm_ctx_profile_enable) is on, launches also create CUDA events the first time a record
+ *    slot is used.
  *  - Device-side failures (a bounded wait that expired) are written to a status
  *    word in the context; read it with nm_ctx_poll_status.
  *  - bias, gamma, beta, scales are fp32 for every activation dtype.
@@ -171,7 +173,8 @@ nm_status nm_linear_pwl(nm_ctx* ctx, const nm_linear_desc* desc, void* stream);
  * Q, K, V: device pointers; element (batch b, token t, head g, channel c) is at
  * base[b*stride_b + t*stride_t + g*d + c], so the three may point into one packed
  * [B*L, 3*heads*d] projection.  out: device [B*L, heads*d], leading dimension
- * heads*d.  dtype F32, BF16 or F16 (fp32 arithmetic inside).
+ * heads*d.  dtype F32, BF16 or F16 (fp32 arithmetic inside).  scale must be positive and finite
+ * (NM_ERR_INVALID_ARG otherwise).
  * algo: 0 = pick; 1 = CUDA-core kernel; 2 = tensor-core kernel that streams K and V and computes
  * Q K^T twice (d = 64, L a multiple of 128); 3 = tensor-core kernel that keeps the whole score block
  * in tensor memory (d = 64, L in {128, 256, 384, 512}). */
@@ -358,9 +361,11 @@ nm_status nm_resnet50_forward_host(nm_ctx* ctx, const nm_conv_params* convs, con
  *
  * Limit: configurations with nm_encoder_workspace_bytes(cfg) > NM_STATIC_WS_BYTES return
  * NM_ERR_WORKSPACE (use nm_encoder_layer with your own workspace for those).
- * First call on a device resolves the array's device address (cudaGetSymbolAddress with that
- * device made current for the moment); make that first call before starting any stream
- * capture.  All calls on a device share the one array and it keeps the previous call's
+ * The array's device address is resolved once, by nm_ctx_create (cudaGetSymbolAddress with the
+ * context's device current; that is also the moment the driver places the array on the device),
+ * and kept in the context, so this call does no set-up of its own on any call, the first
+ * included; NM_ERR_CUDA if that resolution failed.
+ * All calls on a device share the one array and it keeps the previous call's
  * contents: nothing in it needs to start at zero (every buffer is fully written before it is
  * read), but two calls whose kernels overlap on the GPU (different streams, no ordering
  * between them) race on it. */

@@ -59,6 +59,8 @@ def lib():
         _lib.nmo_segment_index.restype = C.c_int32
         _lib.nmo_segment_index.argtypes = [C.POINTER(_Pwl), C.c_float]
         _lib.nmo_num_threads.restype = C.c_int
+        _lib.nmo_antiderivative.restype = C.c_double
+        _lib.nmo_antiderivative.argtypes = [C.c_int, C.c_double]
     return _lib
 
 
@@ -379,8 +381,58 @@ def avgpool_nhwc(x):
     return out
 
 
-def encoder_layer_i8(x, w: dict, q: dict, B, L, h, tables: dict, eps=1e-5):
-    """The int8 evaluation of one encoder layer (Section 5 evaluates INT8 networks): the four weight
+def antiderivative(func, x):
+    """The closed-form integral F (F' = f) that Algorithm 3's segment mean is taken from."""
+    x = _f64(x)
+    f = lib().nmo_antiderivative
+    return np.array([f(func, float(v)) for v in x.ravel()], np.float64).reshape(x.shape)
+
+
+def fake_quant(x, scale, want_codes=False):
+    """Definition-level int8 quantisation in fp64: scale * clamp(rint(x / scale), -127, 127)."""
+    x = _f64(x)
+    y = np.empty_like(x)
+    codes = np.empty(x.shape, np.int8) if want_codes else None
+    lib().nmo_fake_quant(_dp(x), C.c_int64(x.size), C.c_double(float(scale)), _dp(y),
+                         _bp(codes) if want_codes else None)
+    return (y, codes) if want_codes else y
+
+
+def _deq_weight(q, name):
+    return q[name + "_q"].astype(np.float64) * q[name + "_s"].astype(np.float64)[:, None]
+
+
+def encoder_layer_i8(x, w: dict, q: dict, B, L, h, tables: dict, eps=1e-5, want_stages=False):
+    """The int8 evaluation of one encoder layer at DEFINITION level (Section 5 evaluates INT8 networks;
+    the paper fixes no scheme, the reading taken is: weights per output channel, activations per tensor,
+    symmetric).  The tensor entering each of the four weight GEMMs is replaced by the value its int8 code
+    stands for, fq(t) = s * clamp(rint(t / s), -127, 127); everything else is the fp64 layer above.
+    Nothing is rounded to a storage type anywhere:
+        qkv = fq(x) Wqkv^T + b;  a = attention(qkv);  x1 = LN(x + fq(a) Wo^T + bo)
+        g = PWLgelu(fq(x1) W1^T + b1);  y = LN(x1 + fq(g) W2^T + b2)
+    W* are the dequantised int8 weights (code * per-channel scale).  With want_stages the intermediate
+    tensors are returned as well (dict)."""
+    x = _f64(x)
+    H = x.shape[1]
+    d = H // h
+    qkv = linear(fake_quant(x, q["a_x"]), _deq_weight(q, "Wqkv"), w["bqkv"])
+    a = attention(qkv, B, L, h, d, tables["exp"], tables["recip"])
+    z = linear(fake_quant(a, q["a_attn"]), _deq_weight(q, "Wo"), w["bo"], residual=x)
+    x1 = layernorm(z, w["g1"], w["be1"], eps, tables["rsqrt"])
+    g = linear(fake_quant(x1, q["a_x1"]), _deq_weight(q, "W1"), w["b1"], table=tables["gelu"])
+    z2 = linear(fake_quant(g, q["a_g"]), _deq_weight(q, "W2"), w["b2"], residual=x1)
+    y = layernorm(z2, w["g2"], w["be2"], eps, tables["rsqrt"])
+    if want_stages:
+        return y, {"qkv": qkv, "a": a, "z": z, "x1": x1, "g": g, "z2": z2}
+    return y
+
+
+def encoder_layer_i8_storage(x, w: dict, q: dict, B, L, h, tables: dict, eps=1e-5):
+    """A STORAGE MODEL of the int8 layer, not the definition (that is encoder_layer_i8): the same
+    composition with every tensor a bf16 workload keeps in memory rounded to bf16 before it is quantised
+    or reused, and the GELU output requantised from its fp32 value.  The paper fixes none of these
+    rounding points; they describe a workload that stores activations in bf16, and this function exists
+    to tell how much of a GPU-vs-definition difference is storage rounding.  The four weight
     GEMMs take int8 activations (static per-tensor scales q['a_*']) and int8 weights (per-channel scales
     q['W*_s']); everything between them is the fp64 path above.  Composition of the routines in this
     file, in the order of nmo_encoder_layer:

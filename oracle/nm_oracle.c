@@ -25,6 +25,11 @@
  *                       rsqrt and GELU replaced by PWL tables.
  *   nmo_linear_i8       the INT8 evaluation of Section 5: exact integer
  *                       accumulation, then a strict fp32 epilogue.
+ *   nmo_fake_quant      the same evaluation at definition level: a tensor is
+ *                       replaced by the value its int8 code stands for,
+ *                       scale * clamp(rint(x / scale), -127, 127), in fp64.
+ *   nmo_antiderivative  the closed-form integrals Algorithm 3's segment mean
+ *                       uses (exported so that each can be pinned on its own).
  *   nmo_conv2d_nhwc, nmo_maxpool_nhwc, nmo_avgpool_nhwc
  *                       Section 3.1 (convolution is a linear operator) for
  *                       the ResNet-shaped workload; ReLU is a 2-segment table.
@@ -90,6 +95,8 @@ double nmo_exact(int func, double x)
 }
 
 /* antiderivative F with F' = f, for the segment mean of Algorithm 3 */
+static double antiderivative(int func, double x);
+double nmo_antiderivative(int func, double x) { return antiderivative(func, x); }
 static double antiderivative(int func, double x)
 {
     switch (func) {
@@ -439,6 +446,20 @@ void nmo_quantize_i8(const float* x, int64_t count, float inv_scale, int8_t* q)
         if (r > 127.0f) r = 127.0f;
         if (r < -127.0f) r = -127.0f;
         q[i] = (int8_t)r;
+    }
+}
+
+/* Definition-level quantisation (Section 5, INT8 evaluation): the tensor is replaced by the
+ * values its int8 codes stand for.  code = clamp(rint(x / scale), -127, 127), ties to even,
+ * everything in fp64; y = code * scale.  codes may be NULL. */
+void nmo_fake_quant(const double* x, int64_t count, double scale, double* y, int8_t* codes)
+{
+    for (int64_t i = 0; i < count; ++i) {
+        double r = rint(x[i] / scale);
+        if (r > 127.0) r = 127.0;
+        if (r < -127.0) r = -127.0;
+        if (codes) codes[i] = (int8_t)r;
+        y[i] = r * scale;
     }
 }
 

@@ -9,6 +9,13 @@
 
 #include "nm_common.cuh"
 
+// Scratch for nm_encoder_layer_static: a fixed array in the library's own device image.  Every
+// GPU that loads the library carries these NM_STATIC_WS_BYTES until the process exits.
+// In host code the name `nm_static_ws` is only a handle for the runtime, not a device address:
+// the address a kernel may use is the one cudaGetSymbolAddress returns, per device.  nm_ctx_create
+// resolves it (with the context's device current) and keeps it in the context.
+static __device__ __align__(256) unsigned char nm_static_ws[NM_STATIC_WS_BYTES];
+
 namespace {
 
 bool valid_slot(int s) { return s >= 0 && s < NM_NUM_SLOTS; }
@@ -98,6 +105,13 @@ nm_status nm_ctx_create(nm_ctx** out, int device)
         return NM_ERR_CUDA;
     }
     ctx->encode_tiled = fn;
+    {
+        // device address of the library's fixed scratch array on THIS device (the device is current here);
+        // a failure is reported by nm_encoder_layer_static, the only call that needs it
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, nm_static_ws) != cudaSuccess) { p = nullptr; (void)cudaGetLastError(); }
+        ctx->static_ws = p;
+    }
     {
         const char* e = getenv("NM_PDL");   // NM_PDL=0 turns programmatic dependent launch off
         ctx->pdl = (e && e[0] == '0') ? 0 : 1;
@@ -342,6 +356,9 @@ static nm_status attention_dispatch(nm_ctx* ctx, const nm_attn_desc* d, void* st
     if (!nm_aligned16(d->Q) || !nm_aligned16(d->K) || !nm_aligned16(d->V) || !nm_aligned16(d->out))
         return NM_ERR_ALIGNMENT;
     if (d->stride_t < (int64_t)d->heads * d->d || d->stride_b < (int64_t)d->L * d->stride_t) return NM_ERR_SHAPE;
+    // the tensor-core kernels take the row maximum of the raw products and scale it afterwards, which
+    // equals the maximum of the scaled scores only for a positive scale
+    if (!(d->scale > 0.0f) || !isfinite(d->scale)) return NM_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (d->algo == 1) return nm_launch_attention_simt(ctx, d, st);
     // tensor-core kernels: the streaming one (several CTAs per SM, any L that is a multiple of 128) is the
@@ -608,18 +625,6 @@ nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, i
 }  // extern "C"
 
 // ---------------------------------------------------------------- encoder layer without a caller workspace
-//
-// Scratch for nm_encoder_layer_static: a fixed array in the library's own device image.  Every
-// GPU that loads the library carries these NM_STATIC_WS_BYTES until the process exits.
-// In host code the name `nm_static_ws` is only a handle for the runtime, not a device address:
-// the address a kernel may use is the one cudaGetSymbolAddress returns, per device.
-static __device__ __align__(256) unsigned char nm_static_ws[NM_STATIC_WS_BYTES];
-
-namespace {
-constexpr int kMaxDevices = 64;
-void* g_static_ws_ptr[kMaxDevices];   // resolved device address of nm_static_ws, per device
-bool g_static_ws_ready[kMaxDevices];
-}  // namespace
 
 extern "C" nm_status nm_encoder_layer_static(nm_ctx* ctx, const nm_encoder_weights* w, const nm_encoder_cfg* cfg,
                                              const void* x, void* y, void* stream)
@@ -628,24 +633,11 @@ extern "C" nm_status nm_encoder_layer_static(nm_ctx* ctx, const nm_encoder_weigh
     const size_t need = nm_encoder_workspace_bytes(cfg);
     if (need == 0) return NM_ERR_SHAPE;
     if (need > (size_t)NM_STATIC_WS_BYTES) return NM_ERR_WORKSPACE;  // larger layers must bring their own workspace
-    const int dev = ctx->device;
-    if (dev < 0 || dev >= kMaxDevices) return NM_ERR_UNSUPPORTED;
-    if (!g_static_ws_ready[dev]) {
-        // first call on this device: resolve the array's device address with that device current
-        int cur = -1;
-        NM_CUDA_TRY(cudaGetDevice(&cur));
-        if (cur != dev) NM_CUDA_TRY(cudaSetDevice(dev));
-        void* p = nullptr;
-        const cudaError_t e = cudaGetSymbolAddress(&p, nm_static_ws);
-        if (cur != dev) cudaSetDevice(cur);
-        if (e != cudaSuccess || p == nullptr) return NM_ERR_CUDA;
-        g_static_ws_ptr[dev] = p;
-        g_static_ws_ready[dev] = true;
-    }
+    if (!ctx->static_ws) return NM_ERR_CUDA;   // the array's address could not be resolved when the context was made
     // per-launch event records (profiling) would create CUDA events: keep them off in this call
     const int prof = ctx->profiling;
     ctx->profiling = 0;
-    const nm_status s = nm_encoder_layer(ctx, w, cfg, x, y, g_static_ws_ptr[dev], (size_t)NM_STATIC_WS_BYTES, stream);
+    const nm_status s = nm_encoder_layer(ctx, w, cfg, x, y, ctx->static_ws, (size_t)NM_STATIC_WS_BYTES, stream);
     ctx->profiling = prof;
     return s;
 }

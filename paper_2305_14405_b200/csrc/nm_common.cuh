@@ -46,6 +46,7 @@ struct nm_ctx {
     int pdl;                   // launch kernels with programmatic stream serialization (prologue overlap)
     int attn_resident;         // algo 0 prefers the attention kernel with the score block resident in TMEM
     int attn_groups;           // softmax groups per CTA of the streaming attention kernel (1 or 2; 0 = pick)
+    void* static_ws;           // device address of the library's fixed scratch array on this device (or null)
 };
 
 // Brackets one kernel launch with events when profiling is on; counts the launch always.

@@ -102,4 +102,8 @@ def test_attention_argument_errors(nm, ctx):
     with pytest.raises(nm.NmError) as ei:
         ctx.attention_pwl(q, o, 1, 128, 1, 64, exp_slot=12)
     assert ei.value.code == 4
+    for bad_scale in (0.0, -0.125, float("nan"), float("inf")):   # the row maximum is taken before scaling
+        with pytest.raises(nm.NmError) as ei:
+            ctx.attention_pwl(q, o, 1, 128, 1, 64, scale=bad_scale)
+        assert ei.value.code == 1
     ctx.attention_pwl(q, o, 0, 128, 1, 64)     # empty batch: no-op

@@ -1,13 +1,21 @@
-"""GPU parity, int8 encoder layers (config 4 shapes: hidden 1024, 16 heads, FFN 4096, seq 512): the
-four weight GEMMs run as int8 x int8 -> int32 on the tensor cores with an fp32 epilogue; checked per
-layer against the oracle's int8 evaluation on the same int8 weights, scales and bf16 layer input."""
+"""GPU parity, int8 encoder (config 4 shapes: hidden 1024, 16 heads, FFN 4096, seq 512): the four weight
+GEMMs run as int8 x int8 -> int32 on the tensor cores with an fp32 epilogue.
+
+What is asserted, and against what:
+ * stage by stage with the integer decisions shared (every int8 code the GPU feeds a GEMM is handed to the
+   oracle as that GEMM's operand): int32 accumulators, segment numbers and int8 codes bit-exact, every
+   floating-point output within |gpu - oracle| <= 1e-2 + 1e-2*|oracle| on EVERY element;
+ * free-running (the oracle takes its own integer decisions from its own fp64 activations): the share of
+   int8 codes that differ and by how much, and the deviation of a layer / of the whole 24-layer stack from the
+   definition-level oracle (which rounds nothing) and from its bf16-storage model, reported and bounded.
+"""
 import numpy as np
 import pytest
 import torch
 
 import nm_inputs
 import oracle
-from util import assert_close_bf16, load_tables_both, to_np
+from util import assert_close_bf16, load_tables_both, rms_rel, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -19,7 +27,121 @@ def ctx(nm):
     c.close()
 
 
+def _bf16_round(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).bfloat16().float().numpy()
+
+
+def _inv(scale):
+    return float(np.float32(1.0) / np.float32(scale))
+
+
+def test_c4_layer_stage_by_stage_with_shared_integer_decisions(nm, ctx):
+    """One config-4 layer (two sequences) driven stage by stage through the C ABI, so that every tensor
+    exists on the device; each stage is compared with the oracle run on the GPU's own operands of that
+    stage.  The fused layer call must reproduce the staged result bit for bit (its kernels emit the int8
+    codes themselves instead of running the separate quantisation pass)."""
+    from paper_2305_14405_b200.harness import EncoderModel
+    cfg = nm_inputs.with_(nm_inputs.C4, B=2, layers=1)
+    tabs = load_tables_both(ctx, cfg.segments, cfg.ranges())
+    x_np, layers = nm_inputs.encoder_inputs(cfg, seed=4, random_affine=True)
+    w = layers[0]
+    q = nm_inputs.int8_encoder_inputs(cfg, layers)[0]
+    m = EncoderModel(ctx, cfg, layers, quant=[q])
+    d = m.tensors[0]
+    T, H, F, h = cfg.T, cfg.H, cfg.F, cfg.heads
+    dev = "cuda"
+    x = torch.from_numpy(x_np).to(dev).bfloat16()
+
+    def i8(shape):
+        return torch.empty(shape, dtype=torch.int8, device=dev)
+
+    def bf(shape):
+        return torch.full(shape, float("nan"), dtype=torch.bfloat16, device=dev)
+
+    def i32(shape):
+        return torch.full(shape, -12345, dtype=torch.int32, device=dev)
+
+    # ---- the GPU, stage by stage
+    xq = i8((T, H)); ctx.quantize_i8(x, _inv(q["a_x"]), xq)
+    qkv, acc_qkv = bf((T, 3 * H)), i32((T, 3 * H))
+    ctx.linear_pwl(xq, d["Wqkv"], qkv, bias=d["bqkv"], a_scale=q["a_x"], w_scale=d["s_wqkv"], acc_dump=acc_qkv)
+    attn = bf((T, H)); ctx.attention_pwl(qkv, attn, cfg.B, cfg.L, h, cfg.d)
+    aq = i8((T, H)); ctx.quantize_i8(attn, _inv(q["a_attn"]), aq)
+    z, acc_o = bf((T, H)), i32((T, H))
+    ctx.linear_pwl(aq, d["Wo"], z, bias=d["bo"], residual=x, a_scale=q["a_attn"], w_scale=d["s_wo"], acc_dump=acc_o)
+    x1 = bf((T, H)); ctx.layernorm_pwl(z, d["g1"], d["be1"], x1, eps=cfg.eps)
+    x1q = i8((T, H)); ctx.quantize_i8(x1, _inv(q["a_x1"]), x1q)
+    gq, acc_1, idx_1 = i8((T, F)), i32((T, F)), i32((T, F))
+    ctx.linear_pwl(x1q, d["W1"], gq, bias=d["b1"], slot=nm.SLOT_GELU, a_scale=q["a_x1"], w_scale=d["s_w1"],
+                   inv_out_scale=_inv(q["a_g"]), acc_dump=acc_1, idx_dump=idx_1)
+    z2, acc_2 = bf((T, H)), i32((T, H))
+    ctx.linear_pwl(gq, d["W2"], z2, bias=d["b2"], residual=x1, a_scale=q["a_g"], w_scale=d["s_w2"], acc_dump=acc_2)
+    y = bf((T, H)); ctx.layernorm_pwl(z2, d["g2"], d["be2"], y, eps=cfg.eps)
+    ctx.check_device_status()
+    y_fused = m.forward_layer(0, x)
+    ctx.check_device_status()
+    assert torch.equal(y_fused, y), "the fused layer differs from its stages"
+
+    # ---- the oracle, each stage from the GPU's operands of that stage
+    c = lambda t: t.cpu().numpy()
+    f = lambda t: t.float().cpu().numpy()
+    assert np.array_equal(c(xq), oracle.quantize_i8(x_np, q["a_x"]))
+    r = oracle.linear_i8(c(xq), q["Wqkv_q"], q["a_x"], q["Wqkv_s"], w["bqkv"])
+    assert np.array_equal(c(acc_qkv), r["acc"]), "QKV accumulators"
+    assert np.array_equal(f(qkv), _bf16_round(r["y"])), "QKV output (bf16 of the fp32 epilogue value)"
+    assert_close_bf16(f(qkv), r["y"], "C4 stage qkv")
+
+    ref = oracle.attention(f(qkv), cfg.B, cfg.L, h, cfg.d, tabs["exp"], tabs["recip"])
+    assert_close_bf16(f(attn), ref, "C4 stage attention")
+    assert np.array_equal(c(aq), oracle.quantize_i8(f(attn), q["a_attn"]))
+
+    r = oracle.linear_i8(c(aq), q["Wo_q"], q["a_attn"], q["Wo_s"], w["bo"], residual=x_np)
+    assert np.array_equal(c(acc_o), r["acc"]), "out-projection accumulators"
+    assert np.array_equal(f(z), _bf16_round(r["y"]))
+    assert_close_bf16(f(z), r["y"], "C4 stage out-projection + residual")
+
+    ref = oracle.layernorm(f(z), w["g1"], w["be1"], cfg.eps, tabs["rsqrt"])
+    assert_close_bf16(f(x1), ref, "C4 stage LayerNorm 1")
+    assert np.array_equal(c(x1q), oracle.quantize_i8(f(x1), q["a_x1"]))
+
+    r = oracle.linear_i8(c(x1q), q["W1_q"], q["a_x1"], q["W1_s"], w["b1"], table=tabs["gelu"], out_scale=q["a_g"])
+    assert np.array_equal(c(acc_1), r["acc"]), "FFN1 accumulators"
+    assert np.array_equal(c(idx_1), r["idx"]), "FFN1 segment numbers"
+    assert np.array_equal(c(gq), r["q"]), "FFN1 int8 output codes"
+
+    r = oracle.linear_i8(c(gq), q["W2_q"], q["a_g"], q["W2_s"], w["b2"], residual=f(x1))
+    assert np.array_equal(c(acc_2), r["acc"]), "FFN2 accumulators"
+    assert np.array_equal(f(z2), _bf16_round(r["y"]))
+    assert_close_bf16(f(z2), r["y"], "C4 stage FFN2 + residual")
+
+    ref = oracle.layernorm(f(z2), w["g2"], w["be2"], cfg.eps, tabs["rsqrt"])
+    assert_close_bf16(f(y), ref, "C4 stage LayerNorm 2")
+
+    # ---- free-running: the definition-level oracle decides its own codes from its own activations
+    yd, st = oracle.encoder_layer_i8(x_np, w, q, cfg.B, cfg.L, h, tabs, cfg.eps, want_stages=True)
+    for name, gpu_codes, act, scale in (("attention output", aq, st["a"], q["a_attn"]), ("LN1 output", x1q, st["x1"], q["a_x1"]),
+                                        ("GELU output", gq, st["g"], q["a_g"])):
+        _, oc = oracle.fake_quant(act, scale, want_codes=True)
+        diff = np.abs(c(gpu_codes).astype(np.int32) - oc.astype(np.int32))
+        print("free-running codes, %s: %.3f %% differ, max difference %d" % (name, 100 * (diff > 0).mean(), diff.max()))
+        assert (diff > 0).mean() < 0.10 and diff.max() <= 1, name
+    ys = oracle.encoder_layer_i8_storage(x_np, w, q, cfg.B, cfg.L, h, tabs, cfg.eps)
+    got = f(y)
+    for name, ref in (("definition", yd), ("bf16-storage model", ys)):
+        err = np.abs(got - ref)
+        bad = err > 1e-2 + 1e-2 * np.abs(ref)
+        print("free-running layer vs %s: outside bound %d / %d (%.4f %%), max err %.4f, rms(err)/rms(ref) %.5f"
+              % (name, bad.sum(), bad.size, 100 * bad.mean(), err.max(), rms_rel(got, ref)))
+        assert bad.mean() < 1e-2 and rms_rel(got, ref) < 1e-2 and err.max() < 0.1, name
+
+
 def test_c4_int8_layers_sampled(nm, ctx):
+    """Three layers at batch 4, each compared with the oracle started from the GPU's own bf16 layer input,
+    free-running inside the layer.  Codes decided from activations that differ by a bf16 rounding move to
+    a neighbouring code now and then and FFN2 sums 4096 of them, so a fraction of a per cent of the outputs
+    leave the per-element bound (the staged test above holds it for every element): asserted here are
+    >= 99 % of elements inside it, rms(err)/rms(ref) < 1e-2 and max < 0.1, against the definition-level
+    oracle and against its bf16-storage model."""
     from paper_2305_14405_b200.harness import EncoderModel
     cfg = nm_inputs.with_(nm_inputs.C4, B=4, layers=3)
     tabs = load_tables_both(ctx, cfg.segments, cfg.ranges())
@@ -33,41 +155,65 @@ def test_c4_int8_layers_sampled(nm, ctx):
         ctx.check_device_status()
         b = (li + 1) % cfg.B
         xin = to_np(cur[b * L:(b + 1) * L])
-        ref = oracle.encoder_layer_i8(xin, layers[li], quant[li], 1, L, cfg.heads, tabs, cfg.eps)
         got = to_np(nxt[b * L:(b + 1) * L])
-        # Quantised codes are integer decisions taken from floating-point activations.  The oracle takes
-        # them in the workload's storage precision (bf16), yet ~30 % of the attention outputs still differ
-        # from the GPU's by one bf16 ulp (the GPU sums bf16 probabilities in fp32), a few per cent of the
-        # int8 codes downstream move to the neighbouring code, and FFN2 sums 4096 of them: the layer
-        # output carries an error of std ~6e-3 on top of the usual bf16 rounding.  So the per-element
-        # bf16 bound is asserted for 99 % of the elements, with rms and maximum bounds for the rest;
-        # exactness of the int8 arithmetic itself is asserted per GEMM in test_gpu_linear.py.
-        err = np.abs(got - ref)
-        bad = err > 1e-2 + 1e-2 * np.abs(ref)
-        rms = np.sqrt((err ** 2).mean())
-        print("int8 layer %d: max err %.4f, rms %.5f, outside bound %d / %d" % (li, err.max(), rms, bad.sum(), bad.size))
-        assert bad.mean() < 1e-2 and rms < 1e-2 and err.max() < 0.1
+        for name, fn in (("definition", oracle.encoder_layer_i8), ("bf16-storage model", oracle.encoder_layer_i8_storage)):
+            ref = fn(xin, layers[li], quant[li], 1, L, cfg.heads, tabs, cfg.eps)
+            err = np.abs(got - ref)
+            bad = err > 1e-2 + 1e-2 * np.abs(ref)
+            rr = rms_rel(got, ref)
+            print("int8 layer %d vs %s: max err %.4f, rms(err)/rms(ref) %.5f, outside bound %d / %d"
+                  % (li, name, err.max(), rr, bad.sum(), bad.size))
+            assert bad.mean() < 1e-2 and rr < 1e-2 and err.max() < 0.1
         cur = nxt
     y = m.forward(torch.from_numpy(x).cuda().bfloat16())
     assert torch.equal(y, cur)
 
 
-def test_c4_full_size_launch_configuration(nm, ctx):
-    """The 24-layer, batch-16 stack in one call: every launch at its full size; output finite and equal
-    to the layer-by-layer run."""
+def test_c4_full_stack_against_oracle(nm, ctx):
+    """Config 4 as a config: 24 layers with 24 independent weight sets, batch 16, one call, every launch at
+    its full size.  One whole sequence is compared end to end with the definition-level oracle (and with
+    its bf16-storage model); three layers are compared per layer from the GPU's own layer input; the
+    one-call stack equals the layer-by-layer run bit for bit."""
     from paper_2305_14405_b200.harness import EncoderModel
     cfg = nm_inputs.C4
-    load_tables_both(ctx, cfg.segments, cfg.ranges())
-    x, layers = nm_inputs.encoder_inputs(cfg, seed=1, layers=2)
-    layers = [layers[i % 2] for i in range(cfg.layers)]          # 24 layers cycling two weight sets
-    quant2 = nm_inputs.int8_encoder_inputs(cfg, layers[:2])
-    quant = [quant2[i % 2] for i in range(cfg.layers)]
+    tabs = load_tables_both(ctx, cfg.segments, cfg.ranges())
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=1)
+    assert len(layers) == 24 and not np.array_equal(layers[0]["Wqkv"], layers[1]["Wqkv"])
+    quant = nm_inputs.int8_encoder_inputs(cfg, layers)
     m = EncoderModel(ctx, cfg, layers, quant=quant)
     xd = torch.from_numpy(x).cuda().bfloat16()
     y = m.forward(xd)
     ctx.check_device_status()
     assert torch.isfinite(y.float()).all()
+    L = cfg.L
     cur = xd
     for li in range(cfg.layers):
-        cur = m.forward_layer(li, cur)
+        nxt = m.forward_layer(li, cur)
+        if li in (0, 11, 23):
+            b = (5 * li + 2) % cfg.B
+            xin = to_np(cur[b * L:(b + 1) * L])
+            got = to_np(nxt[b * L:(b + 1) * L])
+            ref = oracle.encoder_layer_i8(xin, layers[li], quant[li], 1, L, cfg.heads, tabs, cfg.eps)
+            err = np.abs(got - ref)
+            bad = err > 1e-2 + 1e-2 * np.abs(ref)
+            print("C4 layer %d, sequence %d vs definition: outside bound %d / %d, max err %.4f, rms(err)/rms(ref) %.5f"
+                  % (li, b, bad.sum(), bad.size, err.max(), rms_rel(got, ref)))
+            assert bad.mean() < 1e-2 and rms_rel(got, ref) < 1e-2 and err.max() < 0.1
+        cur = nxt
     assert torch.equal(y, cur)
+    # end to end: sequence 9 through all 24 layers
+    b = 9
+    got = to_np(y[b * L:(b + 1) * L])
+    xin = x[b * L:(b + 1) * L]
+    for name, fn in (("definition", oracle.encoder_layer_i8), ("bf16-storage model", oracle.encoder_layer_i8_storage)):
+        ref = xin
+        for li in range(cfg.layers):
+            ref = fn(ref, layers[li], quant[li], 1, L, cfg.heads, tabs, cfg.eps)
+        err = np.abs(got - ref)
+        bound = 1e-2 + 1e-2 * np.abs(ref)
+        k = np.sqrt(cfg.layers)
+        print("C4 end to end (24 layers) vs %s: outside 1x bound %.4f, outside sqrt(24)x bound %.5f, max err %.4f, "
+              "rms err %.5f, rms(err)/rms(ref) %.5f"
+              % (name, (err > bound).mean(), (err > k * bound).mean(), err.max(), np.sqrt((err ** 2).mean()), rms_rel(got, ref)))
+        # independent per-layer deviations (rms ~5e-3 each, see the per-layer checks) add in quadrature
+        assert rms_rel(got, ref) < np.sqrt(cfg.layers) * 1e-2 and err.max() < 0.5

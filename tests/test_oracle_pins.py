@@ -506,15 +506,16 @@ def test_alg3_bias_correction():
     assert dE[0] < -0.02
 
 
-def test_int8_encoder_layer_against_library_routines():
-    """The int8 evaluation of a layer, rebuilt from library routines only (numpy rint/clip for the
-    quantiser, numpy matmul, torch attention / layer_norm / gelu in fp64, torch bf16 casts) with exact
-    nonlinearities: must agree with the oracle's composition in exact mode."""
+def test_int8_storage_model_layer_against_library_routines():
+    """The bf16-storage model of the int8 layer (not the definition: see the next test), rebuilt from
+    library routines only (numpy rint/clip for the quantiser, numpy matmul, torch attention / layer_norm /
+    gelu in fp64, torch bf16 casts) with exact nonlinearities: must agree with the oracle's composition
+    in exact mode."""
     cfg = nm_inputs.with_(nm_inputs.C4, B=2, L=24, H=64, heads=4, F=128, layers=1)
     x, layers = nm_inputs.encoder_inputs(cfg, seed=5, random_affine=True)
     w = layers[0]
     q = nm_inputs.int8_encoder_inputs(cfg, layers)[0]
-    got = oracle.encoder_layer_i8(x, w, q, cfg.B, cfg.L, cfg.heads, _exact_tables())
+    got = oracle.encoder_layer_i8_storage(x, w, q, cfg.B, cfg.L, cfg.heads, _exact_tables())
 
     def bf(t):
         return torch.from_numpy(np.asarray(t, np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
@@ -540,6 +541,168 @@ def test_int8_encoder_layer_against_library_routines():
     # a code on a rounding boundary may differ between two fp64 summation orders: allow a few elements
     err = np.abs(got - ref)
     assert (err > 1e-9).mean() < 0.02 and np.median(err) < 1e-12
+
+
+# ---------------------------------------------------------------- int8, definition level ----------
+
+def test_fake_quant_is_round_half_even_clamped_and_within_half_a_step():
+    """code = clamp(rint(x / s), -127, 127) in fp64 against numpy, the tie and clamp cases written out,
+    and the defining property |fq(x) - x| <= s / 2 inside the representable range."""
+    s = 0.25
+    x = np.array([0.125, 0.375, 0.625, -0.125, -0.375, 100.0, -100.0, 31.70, 31.80, 0.0])
+    y, codes = oracle.fake_quant(x, s, want_codes=True)
+    assert codes.tolist() == [0, 2, 2, 0, -2, 127, -127, 127, 127, 0]
+    assert np.array_equal(y, codes.astype(np.float64) * s)
+    rng = np.random.default_rng(31)
+    t = rng.standard_normal(5000) * 2.0
+    s = 5.5 / 127.0
+    y, codes = oracle.fake_quant(t, s, want_codes=True)
+    assert np.array_equal(codes, np.clip(np.rint(t / s), -127, 127).astype(np.int8))
+    inside = np.abs(t) <= 127 * s
+    assert np.abs(y - t)[inside].max() <= s / 2 * (1 + 1e-12)
+    assert np.abs(y - t)[inside].max() > s / 2 * 0.98          # the bound is reached: rint, not floor or trunc
+    assert np.all(np.abs(y[~inside]) == 127 * s)
+
+
+def _int8_case(seed=5):
+    cfg = nm_inputs.with_(nm_inputs.C4, B=2, L=24, H=64, heads=4, F=128, layers=1)
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=seed, random_affine=True)
+    q = nm_inputs.int8_encoder_inputs(cfg, layers)[0]
+    return cfg, x.astype(np.float64), layers[0], q
+
+
+def test_int8_layer_definition_against_library_routines():
+    """The definition-level int8 layer (fake-quantise the operand of each of the four GEMMs, round nothing
+    else) rebuilt from library routines only: numpy rint/clip, numpy matmul, torch attention, layer_norm
+    and gelu in fp64, exact nonlinearities.  No bf16 cast anywhere."""
+    cfg, x, w, q = _int8_case()
+    got, st = oracle.encoder_layer_i8(x, w, q, cfg.B, cfg.L, cfg.heads, _exact_tables(), want_stages=True)
+
+    def fq(t, s):
+        return np.clip(np.rint(t / float(s)), -127, 127) * float(s)
+
+    def wdq(name):
+        return q[name + "_q"].astype(np.float64) * q[name + "_s"].astype(np.float64)[:, None]
+
+    H, h, d = cfg.H, cfg.heads, cfg.d
+    ln = lambda t, g, b: torch.nn.functional.layer_norm(torch.from_numpy(t), (H,), torch.from_numpy(g.astype(np.float64)),
+                                                        torch.from_numpy(b.astype(np.float64)), 1e-5).numpy()
+    qkv = fq(x, q["a_x"]) @ wdq("Wqkv").T + w["bqkv"]
+    a = _torch_attention(qkv, cfg.B, cfg.L, h, d)
+    z = fq(a, q["a_attn"]) @ wdq("Wo").T + w["bo"] + x
+    x1 = ln(z, w["g1"], w["be1"])
+    g = torch.nn.functional.gelu(torch.from_numpy(fq(x1, q["a_x1"]) @ wdq("W1").T + w["b1"])).numpy()
+    z2 = fq(g, q["a_g"]) @ wdq("W2").T + w["b2"] + x1
+    ref = ln(z2, w["g2"], w["be2"])
+    assert np.allclose(st["qkv"], qkv, rtol=1e-11, atol=1e-12)
+    # a code that sits on a rounding boundary may fall either way between two fp64 summation orders
+    for name, r in (("a", a), ("z", z), ("x1", x1), ("g", g), ("z2", z2)):
+        e = np.abs(st[name] - r)
+        assert (e > 1e-9).mean() < 0.01 and np.median(e) < 1e-12, name
+    err = np.abs(got - ref)
+    assert (err > 1e-9).mean() < 0.02 and np.median(err) < 1e-12
+
+
+def test_int8_layer_definition_stays_within_the_quantisation_step_of_the_unquantised_layer():
+    """Replacing an operand t by fq(t) moves every entry by at most s/2 (no clamping on these inputs), so a
+    GEMM output moves by at most s/2 * sum_k |W[j,k]|: checked for the first GEMM against the plain fp64
+    linear operator on the same dequantised weights; and the whole layer stays close to the unquantised
+    layer on those weights (int8 with per-tensor scales of ~5 sigma / 127 is a ~1 % perturbation)."""
+    cfg, x, w, q = _int8_case(seed=9)
+    tabs = _exact_tables()
+    y, st = oracle.encoder_layer_i8(x, w, q, cfg.B, cfg.L, cfg.heads, tabs, want_stages=True)
+    wd = {n: q[n + "_q"].astype(np.float64) * q[n + "_s"].astype(np.float64)[:, None] for n in ("Wqkv", "Wo", "W1", "W2")}
+    assert np.abs(x).max() <= 127 * q["a_x"]
+    plain = oracle.linear(x, wd["Wqkv"], w["bqkv"])
+    bound = q["a_x"] / 2 * np.abs(wd["Wqkv"]).sum(axis=1)
+    assert np.all(np.abs(st["qkv"] - plain) <= bound[None, :] * (1 + 1e-9))
+    assert np.abs(st["qkv"] - plain).max() > bound.max() / 50          # and the operand really was quantised
+    w_plain = dict(w)
+    w_plain.update(wd)
+    ref = oracle.encoder_layer(x, w_plain, cfg.B, cfg.L, cfg.heads, tabs)
+    rel = np.sqrt(((y - ref) ** 2).mean()) / np.sqrt((ref ** 2).mean())
+    assert 1e-4 < rel < 3e-2
+
+
+def test_int8_storage_model_differs_from_the_definition_only_by_storage_rounding():
+    """The storage model re-rounds six tensors to bf16 (relative 2^-9 each): its distance from the
+    definition is of that order, not zero and not large."""
+    cfg, x, w, q = _int8_case(seed=11)
+    tabs = _pwl_tables(cfg, 64)
+    xb = nm_inputs.round_to(x.astype(np.float32), "bf16").astype(np.float64)
+    a = oracle.encoder_layer_i8(xb, w, q, cfg.B, cfg.L, cfg.heads, tabs)
+    b = oracle.encoder_layer_i8_storage(xb, w, q, cfg.B, cfg.L, cfg.heads, tabs)
+    rel = np.sqrt(((a - b) ** 2).mean()) / np.sqrt((a ** 2).mean())
+    assert 1e-4 < rel < 2e-2
+
+
+def test_int8_linear_residual_branch_is_one_fp32_add():
+    """y = fl32(fl32(fma(acc, sc, bias)) + residual): the residual branch of the strict fp32 epilogue,
+    against exact rational arithmetic; the integer outputs are untouched by it."""
+    M, N, K = 11, 13, 64
+    Aq = nm_inputs.int8_matrix((M, K), 21)
+    Wq = nm_inputs.int8_matrix((N, K), 22)
+    rng = np.random.default_rng(23)
+    ws = rng.uniform(1e-4, 3e-4, N).astype(np.float32)
+    bias = (0.1 * rng.standard_normal(N)).astype(np.float32)
+    res = rng.standard_normal((M, N)).astype(np.float32)
+    a_scale = np.float32(0.027)
+    t = Table.secant(oracle.GELU, 64, -4.0, 4.0)
+    base = oracle.linear_i8(Aq, Wq, a_scale, ws, bias, None, t)
+    r = oracle.linear_i8(Aq, Wq, a_scale, ws, bias, res, t, out_scale=0.05)
+    assert np.array_equal(r["acc"], base["acc"]) and np.array_equal(r["idx"], base["idx"])
+    inv = np.float32(1.0) / np.float32(0.05)
+    for m in range(M):
+        for j in range(N):
+            ex = Fraction(float(base["y"][m, j])) + Fraction(float(res[m, j]))
+            y = r["y"][m, j]
+            for nb in (np.nextafter(y, np.float32(np.inf)), np.nextafter(y, np.float32(-np.inf))):
+                assert abs(Fraction(float(y)) - ex) <= abs(Fraction(float(nb)) - ex)
+            assert r["q"][m, j] == float(np.clip(np.rint(np.float32(y * inv)), -127, 127))
+    assert np.abs(r["y"] - base["y"]).max() > 0.5           # the residual really was added
+
+
+# ---------------------------------------------------------------- Algorithm 3's integrals ----------
+
+@pytest.mark.parametrize("func,lo,hi", [(oracle.GELU, -4.0, 4.0), (oracle.EXP, -8.0, 0.0), (oracle.RECIP, 0.5, 8.0),
+                                        (oracle.RSQRT, 0.25, 4.0), (oracle.RELU, -1.3, 2.1), (oracle.SQRT, 0.25, 4.0),
+                                        (oracle.IDENTITY, -1.5, 2.5)])
+def test_alg3_antiderivative_against_numerical_quadrature(func, lo, hi):
+    """Every closed-form integral the segment mean of Algorithm 3 is taken from, against adaptive
+    quadrature of the function itself (scipy), on sub-intervals of the range."""
+    import scipy.integrate
+    f = np_f(func)
+    xs = np.linspace(lo, hi, 9)
+    F = oracle.antiderivative(func, xs)
+    for i in range(8):
+        pts = [0.0] if xs[i] < 0.0 < xs[i + 1] else None
+        want, _ = scipy.integrate.quad(lambda v: float(f(np.float64(v))), xs[i], xs[i + 1], points=pts, epsabs=1e-13,
+                                       epsrel=1e-13)
+        assert abs((F[i + 1] - F[i]) - want) <= 1e-11 * max(1.0, abs(want)), (func, i)
+
+
+@pytest.mark.parametrize("func,xs", [(oracle.RSQRT, np.linspace(0.25, 4.0, 9)), (oracle.RELU, np.linspace(-1.2, 1.8, 7)),
+                                     (oracle.IDENTITY, np.linspace(-2.0, 3.0, 6))])
+def test_alg3_bias_correction_rsqrt_relu_identity(func, xs):
+    """dE = mean of f over the segment minus the mean of its secant, against a numerical mean, for the
+    three functions the four-function check above does not cover.  A straight line needs no correction;
+    ReLU only on the segment that straddles 0; a convex function is corrected downwards."""
+    k, b = oracle.secant_points(func, xs)
+    b2, dE = oracle.bias_correct(func, xs, b)
+    n = xs.size - 1
+    f = np_f(func)
+    for i in range(n):
+        x = xs[i] + (xs[i + 1] - xs[i]) * (np.arange(200000) + 0.5) / 200000      # midpoint rule
+        num = (f(x) - (k[i] * x + b[i])).mean()
+        assert abs(dE[i] - num) <= 1e-8 + 1e-6 * abs(num), (func, i)
+    assert np.allclose(b2 - b, dE, rtol=0, atol=1e-15)
+    if func == oracle.IDENTITY:
+        assert np.abs(dE).max() < 1e-15
+    if func == oracle.RELU:
+        straddle = (xs[:-1] < 0) & (xs[1:] > 0)
+        assert straddle.sum() == 1 and dE[straddle][0] < -0.01 and np.abs(dE[~straddle]).max() < 1e-15
+    if func == oracle.RSQRT:
+        assert np.all(dE < 0)
 
 
 def test_maxpool_relu_form_is_the_library_max_pool():

@@ -2,7 +2,8 @@
 (a framework's pool owns the GPU, a serving loop that must not call cudaMalloc, a plug-in that is
 handed only its input and output).  Its scratch is a fixed array inside the library.  The test
 drives it through the C ABI and checks it against nm_encoder_layer with a caller workspace, on
-two calls in a row (the array keeps the previous call's contents), and checks the size limit.
+two calls in a row (the array keeps the previous call's contents), checks that the device's free
+memory is the same before and after the calls (nothing was allocated), and checks the size limit.
 Collected last on purpose: a failure here must not hide any other test."""
 import numpy as np
 import pytest
@@ -28,8 +29,14 @@ def test_static_scratch_layer_matches_workspace_layer(nm):
             x = torch.from_numpy(x_np).cuda().bfloat16()
             want = model.forward_layer(0, x)               # existing entry point, caller workspace
             got = torch.full_like(x, float("nan"))
+            torch.cuda.synchronize()
+            free_before, _ = torch.cuda.mem_get_info()
             ctx.encoder_layer_static(model.structs[0], model.ccfg, x, got)
             torch.cuda.synchronize()
+            free_after, _ = torch.cuda.mem_get_info()
+            # the first call included: the array was placed when the context was created
+            assert free_after == free_before, "call %d changed the device's free memory by %d bytes" % (
+                call, free_before - free_after)
             ctx.check_device_status()
             g, w = got.float().cpu().numpy(), want.float().cpu().numpy()
             assert np.all(np.isfinite(g))
