@@ -318,8 +318,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 #pragma unroll
                 for (int hh = 0; hh < 4; ++hh) {   // 128 keys: the scores span [S_g | O_g]
                     uint32_t r[32];
-                    nm_tmem_ld32_async(t_row + (uint32_t)(hh * 32), r);
-                    nm_tmem_ld_wait32(r);
+                    nm_tmem_ld32_sync(t_row + (uint32_t)(hh * 32), r);
                     if (hh == 3) {   // all of it is in registers: the control warp may overwrite S
                         nm_tc_fence_before();
                         asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
@@ -354,8 +353,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             for (int hh = 0; hh < 2; ++hh) {
                 uint32_t r[32];
                 if (ok) {
-                    nm_tmem_ld32_async(t_row + (uint32_t)(hh * 32), r);
-                    nm_tmem_ld_wait32(r);
+                    nm_tmem_ld32_sync(t_row + (uint32_t)(hh * 32), r);
                 }
                 if (hh == 1) {
                     nm_tc_fence_before();
@@ -426,9 +424,8 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 #pragma unroll
             for (int jj = 0; jj < CH / 16; ++jj) {   // 16 channels at a time, summed over the groups' accumulators
                 uint32_t r0[16], r1[16];
-                nm_tmem_ld16(o_addr + (uint32_t)(jj * 16), r0);
-                if constexpr (NG == 2) nm_tmem_ld16(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
-                nm_tmem_ld_wait();
+                nm_tmem_ld16_sync(o_addr + (uint32_t)(jj * 16), r0);
+                if constexpr (NG == 2) nm_tmem_ld16_sync(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
                 float v[16];
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {

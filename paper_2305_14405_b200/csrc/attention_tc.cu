@@ -219,10 +219,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll 1
             for (int c = h; c < n_pchunks; c += NH) {
                 uint32_t r[64];
-                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64), r);
-                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64 + 32), r + 32);
-                nm_tmem_ld_wait32(r);
-                nm_tmem_ld_wait32(r + 32);
+                nm_tmem_ld32_sync(t_row + (uint32_t)(c * 64), r);
+                nm_tmem_ld32_sync(t_row + (uint32_t)(c * 64 + 32), r + 32);
                 float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
                 for (int i = 0; i < 64; i += 4) {
@@ -252,10 +250,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
                 const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(buf * BQ * ROWB + row * ROWB);
                 uint32_t r[64];
-                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64), r);
-                nm_tmem_ld32_async(t_row + (uint32_t)(c * 64 + 32), r + 32);
-                nm_tmem_ld_wait32(r);
-                nm_tmem_ld_wait32(r + 32);
+                nm_tmem_ld32_sync(t_row + (uint32_t)(c * 64), r);
+                nm_tmem_ld32_sync(t_row + (uint32_t)(c * 64 + 32), r + 32);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {  // 8 keys = one 16-byte chunk of the P row
                     float e[8];

@@ -8,11 +8,21 @@ namespace {
 
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
+// How a convolution reaches the tensor-core kernel.
+enum ConvPath {
+    CONV_DIRECT,    // 1x1, stride 1, no padding: the NHWC activation is the [M, Cin] GEMM operand as it stands
+    CONV_IMPLICIT,  // Cin a multiple of 64: implicit GEMM, one 4-D TMA box of the activation per filter tap
+    CONV_ROWTAP,    // Cin <= 8, kw <= 8 (an RGB first layer): implicit GEMM over a zero-padded 8-channel copy of the
+                    // input, one K-block per filter row: 8 taps x 8 channels = 64 contiguous elements
+    CONV_GATHER     // anything else: explicit gather (im2col) into the workspace, then the GEMM
+};
+
 struct ConvGeom {
     int Ho, Wo, K, Kpad;
     int64_t M;
-    bool direct;      // 1x1, stride 1, no padding: the activation is the GEMM operand
-    bool pad_w;       // weights need their rows padded to Kpad
+    ConvPath path;
+    bool pad_w;       // CONV_GATHER: weights need their rows padded to Kpad
+    int Hp, Wp;       // CONV_ROWTAP: extent of the padded input copy
     size_t a_bytes, w_bytes;
 };
 
@@ -27,10 +37,27 @@ bool conv_geom(const nm_conv_desc* d, ConvGeom* g)
     g->K = d->kh * d->kw * d->Cin;
     g->Kpad = (g->K + 7) & ~7;
     g->M = (int64_t)d->N * g->Ho * g->Wo;
-    g->direct = d->kh == 1 && d->kw == 1 && d->stride == 1 && d->pad == 0 && d->Cin % 8 == 0;
-    g->pad_w = g->Kpad != g->K;
-    g->a_bytes = g->direct ? 0 : align256((size_t)g->M * g->Kpad * 2);
-    g->w_bytes = g->pad_w ? align256((size_t)d->Cout * g->Kpad * 2) : 0;
+    g->pad_w = false;
+    g->Hp = g->Wp = 0;
+    g->a_bytes = g->w_bytes = 0;
+    if (d->kh == 1 && d->kw == 1 && d->stride == 1 && d->pad == 0 && d->Cin % 8 == 0) {
+        g->path = CONV_DIRECT;
+    } else if (d->Cin % 64 == 0 && d->algo != 1) {
+        g->path = CONV_IMPLICIT;
+    } else if (d->Cin <= 8 && d->kw <= 8 && d->algo != 1) {
+        g->path = CONV_ROWTAP;
+        // rows 0 .. (Ho-1)*s + kh - 1 and pixels 0 .. (Wo-1)*s + 7 of the padded copy are read
+        g->Hp = (g->Ho - 1) * d->stride + d->kh;
+        g->Wp = (g->Wo - 1) * d->stride + 8;
+        if (g->Hp < d->H + d->pad) g->Hp = d->H + d->pad;   // (never read, but the copy kernel writes whole rows)
+        g->a_bytes = align256((size_t)d->N * g->Hp * g->Wp * 8 * 2);
+        g->w_bytes = align256((size_t)d->Cout * d->kh * 64 * 2);
+    } else {
+        g->path = CONV_GATHER;
+        g->pad_w = g->Kpad != g->K;
+        g->a_bytes = align256((size_t)g->M * g->Kpad * 2);
+        g->w_bytes = g->pad_w ? align256((size_t)d->Cout * g->Kpad * 2) : 0;
+    }
     return true;
 }
 
@@ -66,10 +93,46 @@ nm_status nm_conv2d_pwl(nm_ctx* ctx, const nm_conv_desc* d, void* workspace, siz
         if (((uintptr_t)workspace & 255u) != 0) return NM_ERR_ALIGNMENT;
     }
     cudaStream_t st = (cudaStream_t)stream;
+    if (g.path == CONV_IMPLICIT || g.path == CONV_ROWTAP) {
+        NmConvTc c;
+        memset(&c, 0, sizeof(c));
+        c.dtype = d->dtype;
+        c.N = d->N; c.Ho = g.Ho; c.Wo = g.Wo; c.Cout = d->Cout;
+        c.bias = d->bias; c.residual = d->residual; c.slot = d->slot; c.res_first = d->res_first; c.out = d->out;
+        c.algo = d->algo;
+        c.flops = 2.0 * (double)g.M * d->Cout * g.K;
+        if (g.path == CONV_IMPLICIT) {
+            c.a_base = d->x;
+            c.a_dim[0] = (uint64_t)d->Cin; c.a_dim[1] = (uint64_t)d->W; c.a_dim[2] = (uint64_t)d->H; c.a_dim[3] = (uint64_t)d->N;
+            c.a_stride[0] = (uint64_t)d->Cin * 2; c.a_stride[1] = (uint64_t)d->W * d->Cin * 2;
+            c.a_stride[2] = (uint64_t)d->H * d->W * d->Cin * 2;
+            c.sw = c.sh = d->stride; c.pw = c.ph = d->pad;
+            c.taps_y = d->kh; c.taps_x = d->kw; c.cblocks = d->Cin / 64;
+            c.w = d->w; c.ldw = g.K; c.Ktot = g.K;
+        } else {
+            // the input with its border and five zero channels written out once (xp), the weights likewise (wp);
+            // output pixel ox then reads the 64 contiguous elements of pixels ox*s .. ox*s + 7 of row oy*s + ky
+            void* xp = workspace;
+            void* wp = (uint8_t*)workspace + g.a_bytes;
+            nm_status s = nm_launch_pad_input(ctx, d->x, xp, d->dtype, d->N, d->H, d->W, d->Cin, d->pad, g.Hp, g.Wp, st);
+            if (s != NM_OK) return s;
+            s = nm_launch_pad_weight(ctx, d->w, wp, d->dtype, d->Cout, d->kh, d->kw, d->Cin, st);
+            if (s != NM_OK) return s;
+            c.a_base = xp;
+            c.a_dim[0] = 64; c.a_dim[1] = (uint64_t)g.Wo; c.a_dim[2] = (uint64_t)g.Hp; c.a_dim[3] = (uint64_t)d->N;
+            c.a_stride[0] = (uint64_t)d->stride * 8 * 2;          // next output pixel: `stride` input pixels on
+            c.a_stride[1] = (uint64_t)g.Wp * 8 * 2;
+            c.a_stride[2] = (uint64_t)g.Hp * g.Wp * 8 * 2;
+            c.sw = 1; c.sh = d->stride; c.pw = 0; c.ph = 0;
+            c.taps_y = d->kh; c.taps_x = 1; c.cblocks = 1;
+            c.w = wp; c.ldw = (int64_t)d->kh * 64; c.Ktot = (int64_t)d->kh * 64;
+        }
+        return nm_launch_conv_tc(ctx, &c, st);
+    }
     const void* A = d->x;
     const void* Wm = d->w;
     int64_t Kg = g.K;
-    if (!g.direct) {
+    if (g.path == CONV_GATHER) {
         void* a_buf = workspace;
         nm_status s = nm_launch_im2col(ctx, d->x, a_buf, d->dtype, d->N, d->H, d->W, d->Cin, d->kh, d->kw, d->stride,
                                        d->pad, g.Ho, g.Wo, g.Kpad, st);

@@ -3,10 +3,10 @@
 // piecewise linear, here a 2-segment table in the GEMM epilogue).
 //
 // A convolution runs as out[M, Cout] = PWL(A[M, K] . W[Cout, K]^T + bias (+ residual)) with
-// M = N*Ho*Wo and K = kh*kw*Cin.  1x1 stride-1 convolutions use the NHWC activation as A
-// directly; every other shape first gathers A (im2col) into the caller's workspace, then
-// calls the same tensor-core linear kernel.  Max-pool and global average pool are small
-// bandwidth-bound kernels.
+// M = N*Ho*Wo and K = kh*kw*Cin on the tensor-core linear kernel.  This file holds the small
+// CUDA-core kernels around it: the zero-padded copies that let a few-channel first layer run as an
+// implicit GEMM, the explicit gather (im2col) kept for channel counts the implicit form does not
+// take, and the pools.
 #include "nm_common.cuh"
 
 namespace {
@@ -101,6 +101,39 @@ __global__ void pad_rows_kernel(const T* __restrict__ w, T* __restrict__ wp, int
         const int64_t r = i / Kpad;
         const int k = (int)(i - r * Kpad);
         wp[i] = k < K ? w[r * K + k] : NmType<T>::from_f(0.f);
+    }
+}
+
+// x [N,H,W,Cin] (Cin <= 8) -> xp [N,Hp,Wp,8]: a border of `pad` zero pixels on the top and left (whatever
+// remains of Hp, Wp on the bottom and right) and zero channels Cin..7; one 16-byte pixel per thread.
+template <typename T>
+__global__ void __launch_bounds__(256) pad_input_kernel(const T* __restrict__ x, T* __restrict__ xp, int Nb, int H,
+                                                        int W, int Cin, int pad, int Hp, int Wp)
+{
+    const int64_t total = (int64_t)Nb * Hp * Wp;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int px = (int)(i % Wp), py = (int)((i / Wp) % Hp), n = (int)(i / ((int64_t)Wp * Hp));
+        const int ix = px - pad, iy = py - pad;
+        T v[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) v[c] = NmType<T>::from_f(0.f);
+        if (ix >= 0 && ix < W && iy >= 0 && iy < H) {
+            const T* src = x + (((int64_t)n * H + iy) * W + ix) * Cin;
+            for (int c = 0; c < Cin; ++c) v[c] = src[c];
+        }
+        *reinterpret_cast<uint4*>(xp + i * 8) = *reinterpret_cast<const uint4*>(v);
+    }
+}
+
+// w [Cout,kh,kw,Cin] (kw <= 8, Cin <= 8) -> wp [Cout,kh,8,8], zero where kx >= kw or c >= Cin
+template <typename T>
+__global__ void pad_weight_kernel(const T* __restrict__ w, T* __restrict__ wp, int Cout, int kh, int kw, int Cin)
+{
+    const int64_t total = (int64_t)Cout * kh * 64;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i & 7), kx = (int)((i >> 3) & 7);
+        const int64_t r = i >> 6;   // (co, ky)
+        wp[i] = (kx < kw && c < Cin) ? w[(r * kw + kx) * Cin + c] : NmType<T>::from_f(0.f);
     }
 }
 
@@ -227,6 +260,26 @@ nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int
         else
             im2col_scalar_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)A, Nb, H, W, Cin, kh, kw, stride, pad, Ho, Wo, Kpad);
     }
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+nm_status nm_launch_pad_input(nm_ctx* ctx, const void* x, void* xp, nm_dtype dt, int Nb, int H, int W, int Cin, int pad,
+                              int Hp, int Wp, cudaStream_t st)
+{
+    const int64_t total = (int64_t)Nb * Hp * Wp;
+    NmLaunchScope scope(ctx, NM_KERNEL_IM2COL, ((double)Nb * H * W * Cin + (double)total * 8) * nm_dtype_size(dt), st);
+    if (dt == NM_F16) pad_input_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)xp, Nb, H, W, Cin, pad, Hp, Wp);
+    else pad_input_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)xp, Nb, H, W, Cin, pad, Hp, Wp);
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+nm_status nm_launch_pad_weight(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, int Cout, int kh, int kw, int Cin,
+                               cudaStream_t st)
+{
+    const int64_t total = (int64_t)Cout * kh * 64;
+    NmLaunchScope scope(ctx, NM_KERNEL_IM2COL, (double)total * 2.0 * nm_dtype_size(dt), st);
+    if (dt == NM_F16) pad_weight_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)w, (__half*)wp, Cout, kh, kw, Cin);
+    else pad_weight_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)wp, Cout, kh, kw, Cin);
     return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
 }
 

@@ -117,11 +117,23 @@ template <> struct NmType<__half> {
     static __device__ __forceinline__ __half from_f(float v) { return __float2half_rn(v); }
 };
 
+// q = clamp(rint(y * inv_scale), -127, 127), ties to even.  Clamped first and rounded in the conversion: the same
+// integer for every input (the bounds are integers), one instruction fewer; NaN gives -127 either way.
 __device__ __forceinline__ int8_t nm_quant_i8(float y, float inv_scale)
 {
-    float r = rintf(y * inv_scale);
-    r = fminf(fmaxf(r, -127.0f), 127.0f);
-    return (int8_t)(int)r;
+    const float v = fminf(fmaxf(y * inv_scale, -127.0f), 127.0f);
+    return (int8_t)__float2int_rn(v);
+}
+// Four such codes packed into one word (byte 0 = a).  The lower bound is applied in fp32, the upper one by the
+// saturating pack instruction: d = (c << 16) | (sat8(a) << 8) | sat8(b).
+__device__ __forceinline__ uint32_t nm_quant_i8x4(float a, float b, float c, float d, float inv_scale)
+{
+    const int ia = __float2int_rn(fmaxf(a * inv_scale, -127.0f)), ib = __float2int_rn(fmaxf(b * inv_scale, -127.0f));
+    const int ic = __float2int_rn(fmaxf(c * inv_scale, -127.0f)), id = __float2int_rn(fmaxf(d * inv_scale, -127.0f));
+    uint32_t hi, w;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(id), "r"(ic), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(ib), "r"(ia), "r"(hi));
+    return w;
 }
 
 // ---------------------------------------------------------------- PTX ---------
@@ -259,6 +271,28 @@ __device__ __forceinline__ void nm_tma_load_3d(void* smem_dst, const CUtensorMap
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(nm_smem_u32(smem_dst)), "l"(tmap), "r"(nm_smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+
+// 4-D tiled load (c0 innermost; NHWC activations as {channel, x, y, image}).  Coordinates beyond the tensor
+// read the fill value (zero), which is how a convolution's border padding is produced.
+__device__ __forceinline__ void nm_tma_load_4d(void* smem_dst, const CUtensorMap* tmap, int c0, int c1, int c2, int c3,
+                                               uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(nm_smem_u32(smem_dst)), "l"(tmap), "r"(nm_smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+// 4-D tiled store shared -> global as one bulk group; parts of the box beyond the tensor's extents are
+// not written.  No coordinate may be negative.
+__device__ __forceinline__ void nm_tma_store_4d(const CUtensorMap* tmap, const void* smem_src, int c0, int c1, int c2,
+                                                int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(tmap),
+                 "r"(nm_smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
 // TMA: 2-D tiled store shared -> global as one bulk group; parts of the box beyond the
@@ -445,6 +479,14 @@ __device__ __forceinline__ void nm_tma_load_2d_2cta(void* smem_dst, const CUtens
         ::"r"(nm_smem_u32(smem_dst)), "l"(tmap), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
         : "memory");
 }
+__device__ __forceinline__ void nm_tma_load_4d_2cta(void* smem_dst, const CUtensorMap* tmap, int c0, int c1, int c2,
+                                                    int c3, uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(nm_smem_u32(smem_dst)), "l"(tmap), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
 __device__ __forceinline__ void nm_tmem_alloc2(uint32_t* smem_slot, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(nm_smem_u32(smem_slot)),
@@ -514,14 +556,19 @@ __host__ __device__ constexpr uint32_t nm_idesc(uint32_t c_fmt, uint32_t ab_fmt,
            ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
-// 32 lanes x 32 consecutive 32-bit columns of tensor memory into registers: thread
-// l of the warp receives row (lane base + l).
-__device__ __forceinline__ void nm_tmem_ld32(uint32_t taddr, uint32_t* r)
+// Tensor-memory reads: 32 lanes x 32 (or 16) consecutive 32-bit columns into registers; thread l of the
+// warp receives row (lane base + l).
+// Load and wait in one statement: the registers are valid when it ends.  (While a tcgen05.ld is in flight
+// its destination registers do not hold the data yet, and a compiler that sees them as ordinary values may
+// copy or spill them before the wait -- a tied in/out operand on a separate wait statement is itself
+// materialised as such a copy -- so the two are never separated.)
+__device__ __forceinline__ void nm_tmem_ld32_sync(uint32_t taddr, uint32_t* r)
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
@@ -529,46 +576,16 @@ __device__ __forceinline__ void nm_tmem_ld32(uint32_t taddr, uint32_t* r)
         : "r"(taddr)
         : "memory");
 }
-// 32 lanes x 16 columns; valid after nm_tmem_ld_wait().
-__device__ __forceinline__ void nm_tmem_ld16(uint32_t taddr, uint32_t* r)
+__device__ __forceinline__ void nm_tmem_ld16_sync(uint32_t taddr, uint32_t* r)
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
-}
-__device__ __forceinline__ void nm_tmem_ld_wait()
-{
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// The same load without the memory clobber, for software-pipelined readers: other
-// loads and stores may move across it.  The destination registers are valid only
-// after nm_tmem_ld_wait32(r), which names them as in/out operands so that no use of
-// r[] can be scheduled above the wait.
-__device__ __forceinline__ void nm_tmem_ld32_async(uint32_t taddr, uint32_t* r)
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr));
-}
-__device__ __forceinline__ void nm_tmem_ld_wait32(uint32_t* r)
-{
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
-                   "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
-                   "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
-                   "+r"(r[29]), "+r"(r[30]), "+r"(r[31]));
 }
 
 // ---------------------------------------------------------------- host --------
@@ -612,6 +629,34 @@ bool nm_attention_tc_supported(const nm_attn_desc* d);
 nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st, int8_t* out_q = nullptr,
                                      float q_inv_scale = 0.f);
 bool nm_attention_stream_supported(const nm_attn_desc* d);
+// Implicit-GEMM convolution on the tensor-core kernel.  The A operand is described as a 4-D view
+// {inner, x, y, image} of the activation (dims in elements, strides in bytes); K-block
+// kb = (ky*taps_x + kx)*cblocks + cb reads the 64 inner elements cb*64.. at x = ox*sw - pw + kx,
+// y = oy*sh - ph + ky for every output pixel (oy, ox) of the tile; W is [Cout, Ktot] with row pitch ldw.
+struct NmConvTc {
+    nm_dtype dtype;
+    const void* a_base;
+    uint64_t a_dim[4];
+    uint64_t a_stride[3];
+    int sw, sh, pw, ph;
+    int taps_y, taps_x, cblocks;
+    const void* w;
+    int64_t ldw, Ktot;
+    int N, Ho, Wo, Cout;
+    const float* bias;
+    const void* residual;
+    int slot, res_first;
+    void* out;
+    int algo;
+    double flops;   // 2 * pixels * Cout * (taps * Cin) of the convolution itself, for the launch records
+};
+nm_status nm_launch_conv_tc(nm_ctx* ctx, const NmConvTc* c, cudaStream_t st);
+// zero-padded copies that let a few-channel first layer run as an implicit GEMM: x [N,H,W,Cin] -> xp [N,Hp,Wp,8]
+// (border of `pad` pixels, channels Cin..7 zero) and w [Cout,kh,kw,Cin] -> wp [Cout,kh,8,8]
+nm_status nm_launch_pad_input(nm_ctx* ctx, const void* x, void* xp, nm_dtype dt, int Nb, int H, int W, int Cin, int pad,
+                              int Hp, int Wp, cudaStream_t st);
+nm_status nm_launch_pad_weight(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, int Cout, int kh, int kw, int Cin,
+                               cudaStream_t st);
 nm_status nm_launch_im2col(nm_ctx* ctx, const void* x, void* A, nm_dtype dt, int Nb, int H, int W, int Cin, int kh,
                            int kw, int stride, int pad, int Ho, int Wo, int Kpad, cudaStream_t st);
 nm_status nm_launch_pad_rows(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, int rows, int K, int Kpad,

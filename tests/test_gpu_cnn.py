@@ -26,14 +26,43 @@ def relu_tables(ctx):
 
 @pytest.mark.parametrize("N,H,W,Cin,Cout,k,stride,pad", [
     (2, 14, 14, 64, 128, 1, 1, 0),      # 1x1: activation used as the GEMM operand directly
-    (2, 14, 14, 64, 64, 3, 1, 1),       # 3x3 gather path
-    (3, 15, 13, 32, 72, 3, 2, 1),       # odd sizes, stride 2
+    (2, 14, 14, 64, 64, 3, 1, 1),       # 3x3, Cin = 64: implicit GEMM
+    (3, 15, 13, 32, 72, 3, 2, 1),       # odd sizes, stride 2, Cin = 32: explicit gather
     (2, 28, 28, 256, 512, 1, 2, 0),     # strided 1x1 (projection shortcut)
-    (2, 40, 40, 3, 64, 7, 2, 3),        # first layer: Cin = 3, K = 147 padded to 152
+    (2, 40, 40, 3, 64, 7, 2, 3),        # first layer: Cin = 3, padded 8-channel copy, one K-block per filter row
     (1, 9, 9, 16, 8, 5, 1, 2),
 ])
 @pytest.mark.parametrize("epi", ["relu", "relu_res", "res_then_relu", "plain"])
 def test_conv2d_parity(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi):
+    _conv_case(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi, nm.ALGO_AUTO)
+
+
+@pytest.mark.parametrize("N,H,W,Cin,Cout,k,stride,pad", [
+    (2, 56, 56, 64, 64, 3, 1, 1),       # stage-1 3x3: 8 x 8 pixel patches of two images, 64-column tile
+    (3, 28, 28, 128, 128, 3, 2, 1),     # strided 3x3 (element-strided boxes), odd image count, 128-column tile
+    (4, 7, 7, 512, 512, 3, 1, 1),       # 7 x 7 images: a patch spans many images
+    (1, 13, 11, 64, 24, 3, 2, 1),       # odd sizes, ragged patches, fewer output channels than a tile
+    (5, 9, 9, 128, 320, 3, 1, 1),       # two column tiles, the second ragged
+    (2, 17, 17, 192, 64, 5, 1, 2),      # 5x5 taps, three channel blocks
+    (2, 33, 29, 3, 32, 7, 2, 3),        # few-channel first layer, odd sizes
+    (2, 20, 20, 3, 16, 3, 1, 1),        # few-channel 3x3, stride 1
+    (1, 12, 12, 8, 64, 5, 1, 0),        # 8 channels, no padding
+])
+@pytest.mark.parametrize("algo", ["pairs", "one_cta"])
+@pytest.mark.parametrize("epi", ["relu_res", "res_then_relu", "plain"])
+def test_conv2d_implicit_gemm_parity(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi, algo):
+    """Shapes that take the implicit-GEMM forms (one TMA box of the activation per filter tap; the padded
+    8-channel copy for a few-channel first layer), with CTA pairs and with one CTA per tile."""
+    _conv_case(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi, nm.ALGO_TC if algo == "pairs" else nm.ALGO_TC_1CTA)
+
+
+def test_conv2d_gather_path_still_agrees(nm, ctx):
+    """algo = 1 keeps the explicit gather and the CUDA-core GEMM: same answer within the tolerance."""
+    _conv_case(nm, ctx, 2, 14, 14, 64, 64, 3, 1, 1, "relu_res", nm.ALGO_SIMT)
+    _conv_case(nm, ctx, 2, 20, 20, 3, 16, 3, 1, 1, "relu", nm.ALGO_SIMT)
+
+
+def _conv_case(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi, algo):
     relu = relu_tables(ctx)
     rng = np.random.default_rng(N * 1000 + H + Cin + k)
     x = nm_inputs.round_to(rng.standard_normal((N, H, W, Cin)).astype(np.float32), "f16")
@@ -47,7 +76,8 @@ def test_conv2d_parity(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi):
     bd = torch.from_numpy(b).cuda()                      # the descriptor holds raw pointers: keep the tensors alive
     rd = torch.from_numpy(res).cuda().half() if res is not None else None
     d = nm.Context.conv_desc(xd, wd, out, stride, pad, bias=bd, residual=rd,
-                             slot=nm.SLOT_NONE if epi == "plain" else nm.SLOT_RELU, res_first=(epi == "res_then_relu"))
+                             slot=nm.SLOT_NONE if epi == "plain" else nm.SLOT_RELU, res_first=(epi == "res_then_relu"),
+                             algo=algo)
     ws_bytes = ctx.conv2d_workspace_bytes(d)
     ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
     ctx.conv2d_pwl(d, ws)
