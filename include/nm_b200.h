@@ -302,7 +302,11 @@ nm_status nm_conv2d_pwl(nm_ctx* ctx, const nm_conv_desc* desc, void* workspace, 
 /* Max pooling, NHWC, window ks x ks, zero-size padding cells ignored (a maximum is itself
  * piecewise linear: max(a,b) = b + ReLU(a-b), Section 3), and global average pooling
  * [N,H,W,C] -> [N,C] (a linear operator, Section 3.1: multiplication by a constant 1/(H*W)
- * matrix; executed on CUDA cores because its operand is channel-contiguous).  C a multiple of 8. */
+ * matrix).  The average runs as a GEMM on the tensor cores: one K-block per position, every
+ * 64-channel block multiplied by the constant matrix (1/(H*W)) * identity, whose entry is rounded
+ * to the storage type (relative 2^-11 for fp16, 2^-8 for bf16); images taller or wider than 256
+ * positions are averaged on CUDA cores instead.  C a multiple of 8.  Calls on one context that
+ * use different H*W or dtypes must not overlap on the GPU (they share the constant matrix). */
 nm_status nm_maxpool2d(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,
                        int32_t C, int32_t ks, int32_t stride, int32_t pad, void* stream);
 nm_status nm_avgpool_global(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype, int32_t N, int32_t H, int32_t W,

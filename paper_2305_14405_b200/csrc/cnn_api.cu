@@ -192,7 +192,31 @@ nm_status nm_avgpool_global(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype,
     if (dtype != NM_F16 && dtype != NM_BF16) return NM_ERR_UNSUPPORTED;
     if (N < 1 || H < 1 || W < 1 || C < 8 || C % 8 != 0) return NM_ERR_SHAPE;
     if (!nm_aligned16(x) || !nm_aligned16(y)) return NM_ERR_ALIGNMENT;
-    return nm_launch_avgpool(ctx, x, y, dtype, N, H * W, C, (cudaStream_t)stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (H > 256 || W > 256) return nm_launch_avgpool(ctx, x, y, dtype, N, H * W, C, st);   // beyond a TMA box: CUDA cores
+    // As a GEMM on the tensor cores: out[n, c] = sum over the H*W positions p and the 64 channels c' of c's block of
+    // x[n, p, c'] * D[c', c], D = (1/HW) * identity.  The implicit-GEMM kernel takes one K-block per position; column
+    // tile t reads channel block t and multiplies by the one constant 64 x 64 matrix D kept in the context.
+    if (ctx->pool_w_hw != H * W || ctx->pool_w_dtype != (int)dtype + 1) {
+        nm_status s = nm_launch_fill_diag(ctx, ctx->d_pool_w, dtype, 1.0f / (float)(H * W), st);
+        if (s != NM_OK) return s;
+        ctx->pool_w_hw = H * W;
+        ctx->pool_w_dtype = (int)dtype + 1;
+    }
+    NmConvTc c;
+    memset(&c, 0, sizeof(c));
+    c.dtype = dtype;
+    c.a_base = x;
+    c.a_dim[0] = (uint64_t)C; c.a_dim[1] = (uint64_t)W; c.a_dim[2] = (uint64_t)H; c.a_dim[3] = (uint64_t)N;
+    c.a_stride[0] = (uint64_t)C * 2; c.a_stride[1] = (uint64_t)W * C * 2; c.a_stride[2] = (uint64_t)H * W * C * 2;
+    c.sw = c.sh = 1; c.pw = c.ph = 0;
+    c.taps_y = H; c.taps_x = W; c.cblocks = 1;
+    c.w = ctx->d_pool_w; c.ldw = 64; c.Ktot = 64;
+    c.N = N; c.Ho = 1; c.Wo = 1; c.Cout = C;
+    c.slot = NM_SLOT_NONE; c.out = y;
+    c.depthwise = 1;
+    c.flops = 2.0 * (double)N * C * H * W;
+    return nm_launch_conv_tc(ctx, &c, st);
 }
 
 // Workspace: four activation buffers of the largest activation (batch x 112 x 112 x 64 =

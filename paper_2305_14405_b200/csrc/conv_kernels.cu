@@ -201,6 +201,13 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const T* __restrict__ x, T
     }
 }
 
+// 64 x 64 matrix with `value` on the diagonal: the constant operand of the average pool run as a GEMM
+template <typename T>
+__global__ void fill_diag_kernel(T* __restrict__ w, float value)
+{
+    for (int i = threadIdx.x; i < 64 * 64; i += blockDim.x) w[i] = NmType<T>::from_f((i >> 6) == (i & 63) ? value : 0.f);
+}
+
 // mean over the HW positions of each image: [N, HW, C] -> [N, C]; 8 channels per thread, fp32 sums
 template <typename T>
 __global__ void __launch_bounds__(256) avgpool_kernel(const T* __restrict__ x, T* __restrict__ y, int Nb, int HW, int C)
@@ -303,6 +310,14 @@ nm_status nm_launch_maxpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, in
         maxpool_kernel<__half><<<grid_for(ctx, total), 256, 0, st>>>((const __half*)x, (__half*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo, relu);
     else
         maxpool_kernel<__nv_bfloat16><<<grid_for(ctx, total), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, Nb, H, W, C, ks, stride, pad, Ho, Wo, relu);
+    return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
+}
+
+nm_status nm_launch_fill_diag(nm_ctx* ctx, void* w, nm_dtype dt, float value, cudaStream_t st)
+{
+    NmLaunchScope scope(ctx, NM_KERNEL_POOL, 64.0 * 64.0 * nm_dtype_size(dt), st);
+    if (dt == NM_F16) fill_diag_kernel<__half><<<1, 256, 0, st>>>((__half*)w, value);
+    else fill_diag_kernel<__nv_bfloat16><<<1, 256, 0, st>>>((__nv_bfloat16*)w, value);
     return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
 }
 

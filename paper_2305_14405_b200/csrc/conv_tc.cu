@@ -52,6 +52,7 @@ nm_status launch(nm_ctx* ctx, const NmConvTc* c, cudaStream_t st)
     cv.sw = c->sw; cv.sh = c->sh; cv.pw = c->pw; cv.ph = c->ph;
     cv.kw_eff = c->taps_x; cv.cblocks = c->cblocks;
     cv.Ho = c->Ho; cv.Nimg = c->N;
+    cv.dw = c->depthwise;
     const int64_t patches = (int64_t)cv.tiles_x * cv.tiles_y * ceil_div(c->N, cv.NB);
     const int64_t m_tiles = TWO ? (patches + 1) / 2 : patches;
     a.M = (int64_t)c->N * c->Ho * c->Wo; a.N = c->Cout; a.K = c->Ktot;
@@ -75,7 +76,8 @@ nm_status launch(nm_ctx* ctx, const NmConvTc* c, cudaStream_t st)
     if (abox[1] > 256 || abox[2] > 256) return NM_ERR_UNSUPPORTED;
     nm_status s = make_tmap4(ctx, &tmA, c->a_base, c->dtype, c->a_dim, c->a_stride, abox, aestr);
     if (s != NM_OK) return s;
-    s = make_tmap(ctx, &tmW, c->w, c->dtype, c->Cout, c->Ktot, c->ldw, B_ROWS);
+    // (depthwise form: W is the one 64 x 64 matrix, whatever the number of output channels)
+    s = make_tmap(ctx, &tmW, c->w, c->dtype, c->depthwise ? 64 : c->Cout, c->Ktot, c->ldw, B_ROWS);
     if (s != NM_OK) return s;
     // output / residual: the 32 tile rows of an epilogue warp are a sub-box of the patch
     const int bh = cv.TH < 32 / cv.TW ? cv.TH : 32 / cv.TW;
@@ -102,7 +104,7 @@ nm_status launch_two(nm_ctx* ctx, const NmConvTc* c, cudaStream_t st)
 template <typename T>
 nm_status launch_sel(nm_ctx* ctx, const NmConvTc* c, cudaStream_t st)
 {
-    if (c->Cout <= 64) return launch_two<T, 64>(ctx, c, st);
+    if (c->Cout <= 64 || c->depthwise) return launch_two<T, 64>(ctx, c, st);
     if (c->Cout <= 128) return launch_two<T, 128>(ctx, c, st);
     return launch_two<T, 256>(ctx, c, st);
 }

@@ -54,6 +54,8 @@ struct ConvDev {
     int sw, sh, pw, ph;     // tap (ky, kx) of output pixel (oy, ox) reads input (oy*sh - ph + ky, ox*sw - pw + kx)
     int kw_eff, cblocks;    // K-block kb = (ky*kw_eff + kx)*cblocks + cb; 64 channels per block
     int Ho, Nimg;           // output rows per image, images
+    int dw;                 // nonzero: "depthwise" form for pooling as a GEMM: column tile nt (64 channels) reads channel
+                            // block nt of the activation at every tap and multiplies by ONE constant 64 x 64 matrix
 };
 
 struct TcArgs {
@@ -279,25 +281,31 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int kb = 0; kb < a.num_k_blocks; ++kb) {
                     if (!__all_sync(0xffffffffu, nm_mbar_wait(&bar_empty[stage], phase ^ 1u, abortp, a.status))) { ok = false; break; }
                     uint8_t* sa = tiles + (size_t)stage * STAGE_BYTES;
-                    int c_w = 0, c_h = 0;
+                    int c_c = 0, c_w = 0, c_h = 0, w_k = kb * BK_ELEMS, w_n = n0;
                     if constexpr (CONV) {
                         const int ky = tap / a.cv.kw_eff, kx = tap - ky * a.cv.kw_eff;
+                        c_c = cb * BK_ELEMS;
                         c_w = pt.ox0 * a.cv.sw - a.cv.pw + kx;
                         c_h = pt.oy0 * a.cv.sh - a.cv.ph + ky;
+                        if (a.cv.dw) {   // pooling: channel block = column tile, one constant matrix for every tap and tile
+                            c_c = (tile % a.num_n_tiles) * BK_ELEMS;
+                            w_k = 0;
+                            w_n = (int)rank * B_ROWS;
+                        }
                     }
                     if (nm_elect_one()) {
                         if constexpr (TWO) {
                             // both CTAs' copies are counted on the leader's barrier
                             const uint32_t full = nm_mapa(nm_smem_u32(&bar_full[stage]), 0);
                             if (rank == 0) nm_mbar_expect_tx(&bar_full[stage], 2 * STAGE_BYTES);
-                            if constexpr (CONV) nm_tma_load_4d_2cta(sa, &tmA, cb * BK_ELEMS, c_w, c_h, pt.img0, full);
+                            if constexpr (CONV) nm_tma_load_4d_2cta(sa, &tmA, c_c, c_w, c_h, pt.img0, full);
                             else nm_tma_load_2d_2cta(sa, &tmA, kb * BK_ELEMS, m0, full);
-                            nm_tma_load_2d_2cta(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, full);
+                            nm_tma_load_2d_2cta(sa + A_BYTES, &tmW, w_k, w_n, full);
                         } else {
                             nm_mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
-                            if constexpr (CONV) nm_tma_load_4d(sa, &tmA, cb * BK_ELEMS, c_w, c_h, pt.img0, &bar_full[stage]);
+                            if constexpr (CONV) nm_tma_load_4d(sa, &tmA, c_c, c_w, c_h, pt.img0, &bar_full[stage]);
                             else nm_tma_load_2d(sa, &tmA, kb * BK_ELEMS, m0, &bar_full[stage]);
-                            nm_tma_load_2d(sa + A_BYTES, &tmW, kb * BK_ELEMS, n0, &bar_full[stage]);
+                            nm_tma_load_2d(sa + A_BYTES, &tmW, w_k, w_n, &bar_full[stage]);
                         }
                     }
                     __syncwarp();

@@ -95,13 +95,14 @@ nm_status nm_ctx_create(nm_ctx** out, int device)
     if (prop.major != 10) { delete ctx; return NM_ERR_UNSUPPORTED; }  // kernels are built for sm_100a only
     if (cudaMalloc(&ctx->d_tables, sizeof(NmTable) * NM_NUM_SLOTS) != cudaSuccess) { delete ctx; return NM_ERR_CUDA; }
     if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess) { cudaFree(ctx->d_tables); delete ctx; return NM_ERR_CUDA; }
+    if (cudaMalloc(&ctx->d_pool_w, 64 * 64 * 2) != cudaSuccess) { cudaFree(ctx->d_tables); cudaFree(ctx->d_status); delete ctx; return NM_ERR_CUDA; }
     cudaMemset(ctx->d_tables, 0, sizeof(NmTable) * NM_NUM_SLOTS);
     cudaMemset(ctx->d_status, 0, sizeof(int));
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
         qres != cudaDriverEntryPointSuccess || !fn) {
-        cudaFree(ctx->d_tables); cudaFree(ctx->d_status); delete ctx;
+        cudaFree(ctx->d_tables); cudaFree(ctx->d_status); cudaFree(ctx->d_pool_w); delete ctx;
         return NM_ERR_CUDA;
     }
     ctx->encode_tiled = fn;
@@ -121,7 +122,7 @@ nm_status nm_ctx_create(nm_ctx** out, int device)
         ctx->attn_groups = (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;   // 0: chosen by sequence length
     }
     ctx->prof = new (std::nothrow) NmProfRecord[NM_PROF_MAX];
-    if (!ctx->prof) { cudaFree(ctx->d_tables); cudaFree(ctx->d_status); delete ctx; return NM_ERR_CUDA; }
+    if (!ctx->prof) { cudaFree(ctx->d_tables); cudaFree(ctx->d_status); cudaFree(ctx->d_pool_w); delete ctx; return NM_ERR_CUDA; }
     *out = ctx;
     return NM_OK;
 }
@@ -136,6 +137,7 @@ nm_status nm_ctx_destroy(nm_ctx* ctx)
     delete[] ctx->prof;
     cudaFree(ctx->d_tables);
     cudaFree(ctx->d_status);
+    cudaFree(ctx->d_pool_w);
     delete ctx;
     return NM_OK;
 }

@@ -47,6 +47,8 @@ struct nm_ctx {
     int attn_resident;         // algo 0 prefers the attention kernel with the score block resident in TMEM
     int attn_groups;           // softmax groups per CTA of the streaming attention kernel (1 or 2; 0 = pick)
     void* static_ws;           // device address of the library's fixed scratch array on this device (or null)
+    void* d_pool_w;            // 64 x 64 matrix (1/HW on the diagonal) of the average pool run as a GEMM; 8 KB
+    int pool_w_hw, pool_w_dtype;   // what d_pool_w currently holds (0 = nothing)
 };
 
 // Brackets one kernel launch with events when profiling is on; counts the launch always.
@@ -648,6 +650,7 @@ struct NmConvTc {
     int slot, res_first;
     void* out;
     int algo;
+    int depthwise;  // pooling as a GEMM: 64-channel column tile nt reads channel block nt; w is one constant 64 x 64 matrix
     double flops;   // 2 * pixels * Cout * (taps * Cin) of the convolution itself, for the launch records
 };
 nm_status nm_launch_conv_tc(nm_ctx* ctx, const NmConvTc* c, cudaStream_t st);
@@ -664,3 +667,5 @@ nm_status nm_launch_pad_rows(nm_ctx* ctx, const void* w, void* wp, nm_dtype dt, 
 nm_status nm_launch_maxpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int H, int W, int C, int ks,
                             int stride, int pad, int Ho, int Wo, cudaStream_t st, int relu_slot = NM_SLOT_NONE);
 nm_status nm_launch_avgpool(nm_ctx* ctx, const void* x, void* y, nm_dtype dt, int Nb, int HW, int C, cudaStream_t st);
+// fills the 64 x 64 matrix `w` with `value` on the diagonal and zero elsewhere
+nm_status nm_launch_fill_diag(nm_ctx* ctx, void* w, nm_dtype dt, float value, cudaStream_t st);

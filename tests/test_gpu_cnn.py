@@ -89,6 +89,21 @@ def _conv_case(nm, ctx, N, H, W, Cin, Cout, k, stride, pad, epi, algo):
     assert_close_bf16(to_np(out), ref, "conv %s" % epi)
 
 
+@pytest.mark.parametrize("N,H,W,C,dtype", [(128, 7, 7, 2048, "f16"), (5, 7, 7, 200, "f16"), (300, 3, 5, 64, "bf16"),
+                                           (2, 1, 300, 72, "f16")])
+def test_avgpool_as_gemm(nm, ctx, N, H, W, C, dtype):
+    """Global average pool as a tensor-core GEMM with the constant matrix (1/HW) * identity (ragged channel
+    blocks, more images than one tile, CTA pairs), and the CUDA-core kernel for a 300-wide image."""
+    rng = np.random.default_rng(N + C)
+    x = nm_inputs.round_to(rng.standard_normal((N, H, W, C)).astype(np.float32) + 0.5, dtype)
+    td = nm_inputs.torch_dtype(dtype)
+    xd = torch.from_numpy(x).cuda().to(td)
+    a = torch.full((N, C), float("nan"), dtype=td, device="cuda")
+    ctx.avgpool_global(xd, a)
+    ctx.check_device_status()
+    assert_close_bf16(to_np(a), oracle.avgpool_nhwc(x), "avgpool %dx%dx%dx%d %s" % (N, H, W, C, dtype))
+
+
 def test_pools_parity(nm, ctx):
     rng = np.random.default_rng(5)
     x = nm_inputs.round_to(rng.standard_normal((3, 23, 17, 64)).astype(np.float32), "f16")
