@@ -195,6 +195,41 @@ typedef struct {
 
 nm_status nm_attention_pwl(nm_ctx* ctx, const nm_attn_desc* desc, void* stream);
 
+/* INT8 attention: both matrix products of attention on int8 tensor cores with int32 accumulation (Section 5
+ * evaluates whole INT8 networks; the paper fixes no scheme, this is the reading taken).  Q, K, V are int8
+ * codes with per-tensor scales s_q, s_k, s_v; the probabilities are int8 codes of the fixed scale 1/127
+ * (they lie in [0, 1]).  Per batch, head and query row i, with every integer exact and every fp32 step one
+ * correctly rounded operation (so the result is defined bit for bit):
+ *     acc_j = <q_i, k_j> (int32);  m = max_j acc_j;  sc = (s_q * s_k) * scale
+ *     x_j = fma((float)acc_j, sc, -((float)m * sc));  e_j = PWL_exp(x_j)   [fp32 index and fma(k, x, b)]
+ *     p_j = clamp(rint(e_j * 127), -127, 127);  sigma = (float)(sum_j p_j) * (1/127)   [integer row sum]
+ *     o_c = sum_j p_j * v_jc (int32);  out_c = ((float)o_c * (s_v * (1/127))) * PWL_recip(sigma)
+ * Element (batch b, token t, head g, channel c) of Q, K, V is at base[b*stride_b + t*stride_t + g*d + c]
+ * (int8, strides in elements = bytes, multiples of 16), so the three may point into one packed [B*L, 3*heads*d]
+ * tensor.  out: device [B*L, heads*d] of out_dtype (BF16 or F32).  d = 64, L a multiple of 128, scale > 0
+ * (NM_ERR_UNSUPPORTED / NM_ERR_INVALID_ARG otherwise: this operator has the tensor-core kernel only).
+ * acc_dump, p_dump: device int32 / int8 [B, heads, L, L] or NULL (the integer scores and the probability codes);
+ * oacc_dump: device int32 [B*L, heads*d] or NULL (the integer P.V), for bit-exact checks. */
+typedef struct {
+    int32_t B, L, heads, d;
+    const int8_t* Q;
+    const int8_t* K;
+    const int8_t* V;
+    int64_t stride_b;
+    int64_t stride_t;
+    float s_q, s_k, s_v;
+    float scale;
+    int32_t exp_slot;
+    int32_t recip_slot;
+    void* out;
+    nm_dtype out_dtype;
+    int32_t* acc_dump;
+    int8_t* p_dump;
+    int32_t* oacc_dump;
+} nm_attn_i8_desc;
+
+nm_status nm_attention_pwl_i8(nm_ctx* ctx, const nm_attn_i8_desc* desc, void* stream);
+
 /* LayerNorm with PWL reciprocal square root (Section 3.2.2 lists sqrt(x) and 1/x;
  * here fused into one rsqrt table):
  *     mu = mean(z);  v = mean((z - mu)^2);  r = PWL_rsqrt(v + eps);  y = (z - mu) * r * gamma + beta

@@ -312,6 +312,31 @@ def linear_i8(Aq, Wq, a_scale, w_scale, bias=None, residual=None, table: Table |
     return {"acc": acc, "idx": idx, "y": y, "q": q}
 
 
+def attention_i8(qkv_q, B, L, h, d, s_q, s_k, s_v, t_exp: Table, t_recip: Table, scale=None, want_dumps=False):
+    """INT8 attention (both matrix products on integers, strict fp32 in between; see nm_oracle.c).
+    qkv_q: packed int8 [B*L, 3*h*d] codes (Q | K | V).  Returns out fp32 [B*L, h*d], or with want_dumps a
+    dict(out, acc int32 [B,h,L,L], p int8 [B,h,L,L], oacc int32 [B*L, h*d])."""
+    qkv_q = np.ascontiguousarray(qkv_q, dtype=np.int8)
+    H = h * d
+    assert qkv_q.shape == (B * L, 3 * H)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    out = np.empty((B * L, H), np.float32)
+    acc = np.empty((B, h, L, L), np.int32) if want_dumps else None
+    pc = np.empty((B, h, L, L), np.int8) if want_dumps else None
+    oacc = np.empty((B * L, H), np.int32) if want_dumps else None
+    base = qkv_q.ctypes.data
+    q = C.cast(base, C.POINTER(C.c_int8))
+    k = C.cast(base + H, C.POINTER(C.c_int8))
+    v = C.cast(base + 2 * H, C.POINTER(C.c_int8))
+    f32 = lambda x: C.c_float(float(np.float32(x)))
+    lib().nmo_attention_i8(q, k, v, C.c_int64(L * 3 * H), C.c_int64(3 * H), C.c_int32(B), C.c_int32(L), C.c_int32(h),
+                           C.c_int32(d), f32(s_q), f32(s_k), f32(s_v), f32(scale), t_exp.ref, t_recip.ref, _fp(out),
+                           _ip(acc) if want_dumps else None, _bp(pc) if want_dumps else None,
+                           _ip(oacc) if want_dumps else None)
+    return {"out": out, "acc": acc, "p": pc, "oacc": oacc} if want_dumps else out
+
+
 def quantize_i8(x, scale):
     x = _f32(x)
     q = np.empty(x.shape, np.int8)

@@ -25,6 +25,9 @@
  *                       rsqrt and GELU replaced by PWL tables.
  *   nmo_linear_i8       the INT8 evaluation of Section 5: exact integer
  *                       accumulation, then a strict fp32 epilogue.
+ *   nmo_attention_i8    the INT8 evaluation extended to the two matrix products of
+ *                       attention (Section 5 evaluates whole INT8 networks): exact
+ *                       integer scores and integer P.V, strict fp32 in between.
  *   nmo_fake_quant      the same evaluation at definition level: a tensor is
  *                       replaced by the value its int8 code stands for,
  *                       scale * clamp(rint(x / scale), -127, 127), in fp64.
@@ -435,6 +438,84 @@ void nmo_linear_i8(const int8_t* Aq, const int8_t* Wq, int64_t M, int64_t N, int
                 q_out[m * N + j] = (int8_t)r;
             }
         }
+    }
+}
+
+/* ---- INT8 attention: both matrix products on integers -------------------------- */
+
+/* Q, K, V are int8 codes with per-tensor scales s_q, s_k, s_v; element (batch bi, token i, head hd,
+ * channel c) at base[bi*stride_b + i*stride_t + hd*d + c].  Per (batch, head, query row i), strict fp32
+ * between the integer parts (every step one correctly rounded fp32 operation, so that a GPU can take the
+ * same integer decisions):
+ *   acc_j  = sum_c Q[i,c]*K[j,c]                          int32, exact
+ *   sc     = (s_q * s_k) * scale                          two fp32 multiplies
+ *   m      = max_j acc_j;  neg = -((float)m * sc)         the row maximum, taken on the integers (sc > 0)
+ *   x_j    = fmaf((float)acc_j, sc, neg)                  scaled score minus the row maximum, one rounding
+ *   e_j    = fmaf(k[s], x_j, b[s]), s = segment of x_j    PWL exponential, fp32 contract
+ *   p_j    = clamp(rintf(e_j * 127), -127, 127)           the probability as an int8 code of scale 1/127
+ *   sigma  = (float)(sum_j p_j) * (1/127)                 the row sum OF THE CODES (an integer sum: exact)
+ *   r      = fmaf(kr[t], sigma, br[t]), t = segment       PWL reciprocal
+ *   o_c    = sum_j p_j*V[j,c]                             int32, exact
+ *   out_c  = ((float)o_c * (s_v * (1/127))) * r           fp32
+ * The paper gives no INT8 scheme; this is the reading taken (probabilities quantised with the fixed scale
+ * 1/127 because they lie in [0, 1], rows normalised by the sum of what is actually multiplied into V).
+ * out is fp32 [B*L, h*d].  acc_dump / p_dump / oacc_dump (any may be NULL): scores [B,h,L,L] int32, codes
+ * [B,h,L,L] int8, integer P.V [B*L, h*d] int32. */
+void nmo_attention_i8(const int8_t* Q, const int8_t* Kp, const int8_t* V, int64_t stride_b, int64_t stride_t,
+                      int32_t B, int32_t L, int32_t h, int32_t d, float s_q, float s_k, float s_v, float scale,
+                      const nmo_pwl* t_exp, const nmo_pwl* t_recip, float* out, int32_t* acc_dump,
+                      int8_t* p_dump, int32_t* oacc_dump)
+{
+    const float sc = (s_q * s_k) * scale;
+    const float inv127 = 1.0f / 127.0f;
+    const float c1 = s_v * inv127;
+    int64_t rows = (int64_t)B * h * L;
+#pragma omp parallel
+    {
+        int32_t* acc = (int32_t*)malloc(sizeof(int32_t) * (size_t)L);
+        int8_t* p = (int8_t*)malloc((size_t)L);
+#pragma omp for schedule(static)
+        for (int64_t row = 0; row < rows; ++row) {
+            int64_t bi = row / ((int64_t)h * L);
+            int64_t hd = (row / L) % h;
+            int64_t i = row % L;
+            const int8_t* q = Q + bi * stride_b + i * stride_t + hd * d;
+            int32_t m = INT32_MIN;
+            for (int64_t j = 0; j < L; ++j) {
+                const int8_t* kk = Kp + bi * stride_b + j * stride_t + hd * d;
+                int32_t a = 0;
+                for (int c = 0; c < d; ++c) a += (int32_t)q[c] * (int32_t)kk[c];
+                acc[j] = a;
+                if (a > m) m = a;
+            }
+            float neg = -((float)m * sc);
+            int32_t isum = 0;
+            for (int64_t j = 0; j < L; ++j) {
+                float x = fmaf((float)acc[j], sc, neg);
+                int32_t s = nmo_segment_index(t_exp, x);
+                float e = fmaf(t_exp->k[s], x, t_exp->b[s]);
+                float rr = rintf(e * 127.0f);
+                if (rr > 127.0f) rr = 127.0f;
+                if (!(rr >= -127.0f)) rr = -127.0f;   /* also NaN, as in the quantiser above */
+                p[j] = (int8_t)rr;
+                isum += p[j];
+            }
+            float sigma = (float)isum * inv127;
+            int32_t t = nmo_segment_index(t_recip, sigma);
+            float r = fmaf(t_recip->k[t], sigma, t_recip->b[t]);
+            float* o = out + (bi * L + i) * ((int64_t)h * d) + hd * d;
+            for (int c = 0; c < d; ++c) {
+                int32_t oa = 0;
+                for (int64_t j = 0; j < L; ++j)
+                    oa += (int32_t)p[j] * (int32_t)V[bi * stride_b + j * stride_t + hd * d + c];
+                if (oacc_dump) oacc_dump[(bi * L + i) * ((int64_t)h * d) + hd * d + c] = oa;
+                o[c] = ((float)oa * c1) * r;
+            }
+            if (acc_dump) memcpy(acc_dump + row * L, acc, sizeof(int32_t) * (size_t)L);
+            if (p_dump) memcpy(p_dump + row * L, p, (size_t)L);
+        }
+        free(acc);
+        free(p);
     }
 }
 

@@ -30,7 +30,7 @@ EXPORTS = [
     "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
     "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_maxpool2d_pwl", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
     "nm_resnet50_forward", "nm_resnet50_forward_host", "nm_pwl_table_build_elastic",
-    "nm_selftest_bounded_wait",
+    "nm_selftest_bounded_wait", "nm_attention_pwl_i8",
 ]
 KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc",
                 "im2col", "pool")
@@ -57,6 +57,14 @@ class AttnDesc(C.Structure):
                 ("Q", C.c_void_p), ("K", C.c_void_p), ("V", C.c_void_p), ("stride_b", C.c_int64),
                 ("stride_t", C.c_int64), ("scale", C.c_float), ("exp_slot", C.c_int32), ("recip_slot", C.c_int32),
                 ("out", C.c_void_p), ("algo", C.c_int32)]
+
+
+class AttnI8Desc(C.Structure):
+    _fields_ = [("B", C.c_int32), ("L", C.c_int32), ("heads", C.c_int32), ("d", C.c_int32), ("Q", C.c_void_p),
+                ("K", C.c_void_p), ("V", C.c_void_p), ("stride_b", C.c_int64), ("stride_t", C.c_int64),
+                ("s_q", C.c_float), ("s_k", C.c_float), ("s_v", C.c_float), ("scale", C.c_float),
+                ("exp_slot", C.c_int32), ("recip_slot", C.c_int32), ("out", C.c_void_p), ("out_dtype", C.c_int),
+                ("acc_dump", C.c_void_p), ("p_dump", C.c_void_p), ("oacc_dump", C.c_void_p)]
 
 
 class EncoderWeights(C.Structure):
@@ -119,6 +127,7 @@ def load():
                                  C.c_void_p]
     lib.nm_linear_pwl.argtypes = [C.c_void_p, C.POINTER(LinearDesc), C.c_void_p]
     lib.nm_attention_pwl.argtypes = [C.c_void_p, C.POINTER(AttnDesc), C.c_void_p]
+    lib.nm_attention_pwl_i8.argtypes = [C.c_void_p, C.POINTER(AttnI8Desc), C.c_void_p]
     lib.nm_layernorm_pwl.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                      C.c_int32, C.c_float, C.c_int32, C.c_int, C.c_void_p]
     lib.nm_layernorm_pwl_sqrt_recip.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
@@ -318,6 +327,24 @@ class Context:
         a.out = out.data_ptr()
         a.algo = algo
         _check(self._lib.nm_attention_pwl(self._h, C.byref(a), _stream(stream)), "nm_attention_pwl")
+
+    def attention_pwl_i8(self, qkv_q, out, B, L, heads, d, s_q, s_k, s_v, scale=None, exp_slot=SLOT_EXP,
+                         recip_slot=SLOT_RECIP, acc_dump=None, p_dump=None, oacc_dump=None, stream=None):
+        """qkv_q: packed int8 [B*L, 3*heads*d] codes (Q | K | V); out: [B*L, heads*d] bf16 or fp32."""
+        H = heads * d
+        a = AttnI8Desc()
+        a.B, a.L, a.heads, a.d = B, L, heads, d
+        base = qkv_q.data_ptr()
+        a.Q, a.K, a.V = base, base + H, base + 2 * H
+        a.stride_b, a.stride_t = L * qkv_q.stride(0), qkv_q.stride(0)
+        a.s_q, a.s_k, a.s_v = float(s_q), float(s_k), float(s_v)
+        a.scale = float(scale) if scale is not None else float(d) ** -0.5
+        a.exp_slot, a.recip_slot = exp_slot, recip_slot
+        a.out, a.out_dtype = out.data_ptr(), dtype_of(out)
+        a.acc_dump = acc_dump.data_ptr() if acc_dump is not None else None
+        a.p_dump = p_dump.data_ptr() if p_dump is not None else None
+        a.oacc_dump = oacc_dump.data_ptr() if oacc_dump is not None else None
+        _check(self._lib.nm_attention_pwl_i8(self._h, C.byref(a), _stream(stream)), "nm_attention_pwl_i8")
 
     def layernorm_pwl(self, x, gamma, beta, y, eps=1e-5, rsqrt_slot=SLOT_RSQRT, stream=None):
         rows, H = x.shape

@@ -382,6 +382,30 @@ static nm_status attention_dispatch(nm_ctx* ctx, const nm_attn_desc* d, void* st
     return nm_launch_attention_simt(ctx, d, st);
 }
 
+nm_status nm_attention_pwl_i8(nm_ctx* ctx, const nm_attn_i8_desc* d, void* stream)
+{
+    if (!ctx || !d) return NM_ERR_INVALID_ARG;
+    if (d->B < 0 || d->L < 0 || d->heads < 0 || d->d < 0) return NM_ERR_SHAPE;
+    nm_status s = need_table(ctx, d->exp_slot);
+    if (s != NM_OK) return s;
+    s = need_table(ctx, d->recip_slot);
+    if (s != NM_OK) return s;
+    if (d->B == 0 || d->L == 0 || d->heads == 0 || d->d == 0) return NM_OK;
+    if (!d->Q || !d->K || !d->V || !d->out) return NM_ERR_INVALID_ARG;
+    if (d->out_dtype != NM_BF16 && d->out_dtype != NM_F32) return NM_ERR_UNSUPPORTED;
+    if (!(d->scale > 0.0f) || !isfinite(d->scale) || !(d->s_q > 0.0f) || !(d->s_k > 0.0f) || !(d->s_v > 0.0f))
+        return NM_ERR_INVALID_ARG;
+    if (!nm_aligned16(d->Q) || !nm_aligned16(d->K) || !nm_aligned16(d->V) || !nm_aligned16(d->out) ||
+        !nm_aligned16(d->acc_dump) || !nm_aligned16(d->p_dump) || !nm_aligned16(d->oacc_dump))
+        return NM_ERR_ALIGNMENT;
+    if (d->stride_t % 16 != 0 || d->stride_b % 16 != 0) return NM_ERR_ALIGNMENT;
+    if (d->stride_t < (int64_t)d->heads * d->d || d->stride_b < (int64_t)d->L * d->stride_t) return NM_ERR_SHAPE;
+    if (d->d != 64 || d->L % 128 != 0) return NM_ERR_UNSUPPORTED;
+    // the replicated exp table must fit beside the tiles
+    if ((size_t)(ctx->h_tables[d->exp_slot].n + 1) * 16 * sizeof(float2) > 16 * 1024) return NM_ERR_UNSUPPORTED;
+    return nm_launch_attention_i8(ctx, d, (cudaStream_t)stream);
+}
+
 // q != nullptr: the kernel also writes the int8 codes of its (rounded) output, scale 1/q_inv_scale
 static nm_status layernorm_checked(nm_ctx* ctx, const void* x, const float* gamma, const float* beta, void* y,
                                    int64_t rows, int32_t H, float eps, int32_t rsqrt_slot, nm_dtype dtype, void* stream,

@@ -631,6 +631,7 @@ bool nm_attention_tc_supported(const nm_attn_desc* d);
 nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st, int8_t* out_q = nullptr,
                                      float q_inv_scale = 0.f);
 bool nm_attention_stream_supported(const nm_attn_desc* d);
+nm_status nm_launch_attention_i8(nm_ctx* ctx, const nm_attn_i8_desc* d, cudaStream_t st);
 // Implicit-GEMM convolution on the tensor-core kernel.  The A operand is described as a 4-D view
 // {inner, x, y, image} of the activation (dims in elements, strides in bytes); K-block
 // kb = (ky*taps_x + kx)*cblocks + cb reads the 64 inner elements cb*64.. at x = ox*sw - pw + kx,

@@ -755,3 +755,82 @@ def test_resnet50_composition_against_torch():
     ref = (y.mean(dim=(2, 3)) @ torch.from_numpy(fc_w.astype(np.float64)).T + torch.from_numpy(fc_b.astype(np.float64))).numpy()
     assert np.allclose(got, ref, rtol=1e-10, atol=1e-9)
     assert len(convs) == 53 and sum(c["w"].size for c in convs) + fc_w.size > 23e6   # ResNet-50's ~23.5 M conv weights
+
+
+# ---------------------------------------------------------------- int8 attention ----------
+
+def _i8_attn_case(B=2, L=24, h=2, d=16, seed=41):
+    rng = np.random.default_rng(seed)
+    qkv = rng.standard_normal((B * L, 3 * h * d)).astype(np.float32)
+    s = np.float32(4.0 / 127.0)
+    codes = np.clip(np.rint(qkv / s), -127, 127).astype(np.int8)
+    return codes, s
+
+
+def test_int8_attention_integer_parts_are_exact_and_fp32_steps_are_single_roundings():
+    """Scores and P.V against int64 matmuls; every fp32 step against exact rational arithmetic; the codes
+    against numpy rint/clip; the row sum is the integer sum of the codes."""
+    B, L, h, d = 2, 24, 2, 16
+    codes, s = _i8_attn_case(B, L, h, d)
+    H = h * d
+    te = Table.secant(oracle.EXP, 64, -8.0, 0.0)
+    tr = Table.secant(oracle.RECIP, 64, 1.0, float(L))
+    r = oracle.attention_i8(codes, B, L, h, d, s, s, s, te, tr, want_dumps=True)
+    scale = np.float32(1.0 / np.sqrt(d))
+    sc = np.float32(np.float32(s * s) * scale)
+    inv127 = np.float32(1.0) / np.float32(127.0)
+    c1 = np.float32(s * inv127)
+    def near(y, ex):       # y is the float nearest to the exact rational ex
+        for nb in (np.nextafter(y, np.float32(np.inf)), np.nextafter(y, np.float32(-np.inf))):
+            assert abs(Fraction(float(y)) - ex) <= abs(Fraction(float(nb)) - ex)
+    for b in range(B):
+        for g in range(h):
+            q = codes[b * L:(b + 1) * L, g * d:(g + 1) * d].astype(np.int64)
+            k = codes[b * L:(b + 1) * L, H + g * d:H + (g + 1) * d].astype(np.int64)
+            v = codes[b * L:(b + 1) * L, 2 * H + g * d:2 * H + (g + 1) * d].astype(np.int64)
+            acc = q @ k.T
+            assert np.array_equal(r["acc"][b, g], acc.astype(np.int32))
+            p = r["p"][b, g].astype(np.int64)
+            assert np.array_equal(r["oacc"][b * L:(b + 1) * L, g * d:(g + 1) * d], (p @ v).astype(np.int32))
+            for i in range(0, L, 5):
+                m = int(acc[i].max())
+                neg = np.float32(-(np.float32(m) * sc))
+                near(neg, -(Fraction(m) * Fraction(float(sc))))
+                for j in range(0, L, 3):
+                    x = np.float32(float(Fraction(int(acc[i, j])) * Fraction(float(sc)) + Fraction(float(neg))))
+                    ex = Fraction(int(acc[i, j])) * Fraction(float(sc)) + Fraction(float(neg))
+                    for nb in (np.nextafter(x, np.float32(np.inf)), np.nextafter(x, np.float32(-np.inf))):
+                        if abs(Fraction(float(nb)) - ex) < abs(Fraction(float(x)) - ex):
+                            x = nb
+                    e, _ = oracle.pwl_eval_f32(te, np.array([x], np.float32))
+                    assert p[i, j] == int(np.clip(np.rint(np.float32(e[0] * np.float32(127.0))), -127, 127))
+                sigma = np.float32(np.float32(int(p[i].sum())) * inv127)
+                rr, _ = oracle.pwl_eval_f32(tr, np.array([sigma], np.float32))
+                for c in range(0, d, 4):
+                    oa = int((p[i] * v[:, c]).sum())
+                    want = np.float32(np.float32(np.float32(oa) * c1) * rr[0])
+                    assert r["out"][b * L + i, g * d + c] == want
+
+
+def test_int8_attention_approaches_float_attention():
+    """With fine tables (256 segments: table error ~1e-3), int8 attention equals textbook attention on the
+    dequantised operands up to the quantisation of the probabilities (step 1/127, at most 1/254 off per key):
+    the output moves by at most sum_j |v_j| / 254 per row before normalisation; and the rows of codes are
+    normalised by their own sum, so a row of identical scores returns the mean of V as float attention does."""
+    B, L, h, d = 1, 32, 2, 16
+    codes, s = _i8_attn_case(B, L, h, d, seed=43)
+    te, tr = Table.secant(oracle.EXP, 256, -16.0, 0.0), Table.secant(oracle.RECIP, 256, 0.5, 33.0)
+    out = oracle.attention_i8(codes, B, L, h, d, s, s, s, te, tr).astype(np.float64)
+    deq = codes.astype(np.float64) * float(s)
+    ref = _torch_attention(deq, B, L, h, d)
+    H = h * d
+    vabs = np.abs(deq[:, 2 * H:]).reshape(L, h, d).sum(axis=0)          # sum_j |v_j| per (head, channel)
+    # normalised by sigma >= 1 (the maximum element has code 127); a loose but rigorous envelope
+    bound = (vabs / 254.0 + np.abs(ref).reshape(L, h, d).max(axis=0) * L / 254.0).reshape(1, H)
+    assert np.all(np.abs(out - ref) <= bound + 5e-3 * np.abs(ref).max())
+    assert np.abs(out - ref).max() < 0.05 and np.abs(out - ref).max() > 1e-5      # close, and really quantised
+    z = codes.copy()
+    z[:, :2 * H] = 0                                                            # all scores equal
+    out = oracle.attention_i8(z, B, L, h, d, s, s, s, te, tr).astype(np.float64)
+    want = (z[:, 2 * H:].astype(np.float64) * float(s)).mean(axis=0, keepdims=True)
+    assert np.allclose(out, np.repeat(want, L, axis=0), rtol=2e-3, atol=1e-4)     # the 1/x table's own error
