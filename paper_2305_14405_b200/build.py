@@ -51,8 +51,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
             list(ex.map(run, jobs))
     if jobs or force or not os.path.exists(SO) or any(os.path.getmtime(o) > os.path.getmtime(SO) for o in objs):
         tmp = SO + ".tmp.%d" % os.getpid()
-        run([NVCC, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
-        os.replace(tmp, SO)
+        try:
+            run([NVCC, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
+            os.replace(tmp, SO)
+        finally:
+            if os.path.exists(tmp):
+                os.remove(tmp)
     return SO
 
 
