@@ -12,6 +12,10 @@
 // shared memory per softmax group (plus Q and the table): two or three CTAs fit on an SM and one
 // CTA's loads, MMAs and hand-offs overlap the others' arithmetic.  Any L that is a multiple of 128.
 //
+// The 16-bit P tile of the one-group form never touches shared memory: the softmax warps write it to 32 further
+// tensor-memory columns (tcgen05.st) and P V takes its A operand from there; the shared-memory pipe, which the
+// table lookups load most, loses the tile's stores and the tensor core's reads of it.
+//
 // A group is one control warp and four softmax warps, an independent pipeline that owns 128
 // tensor-memory columns [S_g | O_g], two K stages, a V stage and a P tile.  A CTA has NG = 1 or 2
 // groups (template parameter); with two, the groups split the keys: in sweep 1 group g takes the
@@ -72,6 +76,32 @@ template <> struct AT<__half> {
     }
 };
 
+// 16 packed words of this thread's row into 16 consecutive tensor-memory columns (the mirror of the 16-column read)
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r)
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait()
+{
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+// D (+)= A B with the A operand in tensor memory: row m of A in lane m, elements 2c and 2c + 1 of the row in the
+// low and high half of column c (16 elements = 8 columns per instruction)
+__device__ __forceinline__ void mma_f16_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 __device__ __forceinline__ float max3f(float a, float b, float c)
 {
     float d;
@@ -93,11 +123,17 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     constexpr int NSOFT = 128 * NG;            // softmax threads
     constexpr uint32_t GRP_COLS = 128;    // tensor-memory columns of a group
     constexpr uint32_t O_OFF = 64;        // O_g within the group's columns
+    // One group per CTA: the 16-bit P tile goes through tensor memory (a second allocation of 32 columns: 64 keys,
+    // two per column) and is the A operand of P V from there; three CTAs hold 3 x (128 + 32) of the SM's 512
+    // columns.  That takes the P tile's stores, its reads by the tensor core and the proxy fence off the shared-
+    // memory pipe, which the table lookups load most.  With two groups the columns do not suffice (2 CTAs x 320).
+    constexpr bool PT = NG == 1;
+    constexpr uint32_t P_COLS = 32;
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_q, bar_drain[NG];
     __shared__ uint64_t bar_k_full[NG][2], bar_k1_full[NG][2], bar_v_full[NG], bar_s_full[NG], bar_p_empty[NG];
-    __shared__ uint32_t tmem_slot;
+    __shared__ uint32_t tmem_slot, tmem_slot_p;
     __shared__ int abort_flag;
     __shared__ float s_red[NG][BQ];
 
@@ -157,6 +193,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     }
     if (warp == NG - 1) {
         nm_tmem_alloc(&tmem_slot, TMEM_COLS);
+        if constexpr (PT) nm_tmem_alloc(&tmem_slot_p, P_COLS);
         nm_tmem_relinquish();
     }
     if (warp >= NG) {
@@ -170,6 +207,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     __syncthreads();
     nm_tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    const uint32_t tmem_p = PT ? tmem_slot_p : 0u;
     volatile int* abortp = &abort_flag;
     nm_grid_launch_dependents();   // the next kernel may start its set-up
     nm_grid_dependency_wait();     // Q, K, V come from the previous kernel
@@ -256,9 +294,11 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const uint32_t v_addr = nm_smem_u32(my_v);
                 if (nm_elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
-                        nm_mma_f16(my_tmem + O_OFF, pdesc + 2 * k, nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB)),
-                                   IDESC_PV, (j | k) != 0);
+                    for (int k = 0; k < 4; ++k) {   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
+                        const uint64_t vdesc = nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB));
+                        if constexpr (PT) mma_f16_a_tmem(my_tmem + O_OFF, tmem_p + (uint32_t)(8 * k), vdesc, IDESC_PV, (j | k) != 0);
+                        else nm_mma_f16(my_tmem + O_OFF, pdesc + 2 * k, vdesc, IDESC_PV, (j | k) != 0);
+                    }
                     nm_tc_commit(&bar_p_empty[gi]);
                 }
                 __syncwarp();
@@ -344,6 +384,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         const float neg_ms = -(m * a.scale);
         float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
         const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(g2 * PBUF + row * ROWB);
+        const uint32_t p_row = tmem_p + ((uint32_t)(q * 32) << 16);   // this warp's lane quarter of the P columns
         // ---- sweep 2: e = PWL_exp(s - m), row sum, P tiles
 #pragma unroll 1
         for (int j = 0; j < half; ++j) {
@@ -389,17 +430,27 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     wait_all(&bar_p_empty[g2], (uint32_t)((j - 1) & 1));
                 }
                 if (ok) {
+                    if constexpr (PT) {
+                        if (hh == 0 && j >= 1) nm_tc_fence_after();   // ordered after the P V that read the columns
+                        tmem_st16(p_row + (uint32_t)(hh * 16), pk);   // keys 32 hh .. 32 hh + 31 of this thread's row
+                    } else {
 #pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        // chunk index is XORed with the row (128-byte swizzle of the K-major P tile)
-                        const uint32_t addr = prow + (uint32_t)(((hh * 4 + jj) ^ (row & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pk[jj * 4]), "r"(pk[jj * 4 + 1]),
-                                     "r"(pk[jj * 4 + 2]), "r"(pk[jj * 4 + 3])
-                                     : "memory");
+                        for (int jj = 0; jj < 4; ++jj) {
+                            // chunk index is XORed with the row (128-byte swizzle of the K-major P tile)
+                            const uint32_t addr = prow + (uint32_t)(((hh * 4 + jj) ^ (row & 7)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pk[jj * 4]), "r"(pk[jj * 4 + 1]),
+                                         "r"(pk[jj * 4 + 2]), "r"(pk[jj * 4 + 3])
+                                         : "memory");
+                        }
                     }
                 }
             }
-            nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
+            if constexpr (PT) {
+                tmem_st_wait();          // the P columns are written
+                nm_tc_fence_before();
+            } else {
+                nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
+            }
             asm volatile("bar.arrive %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");
         }
         float sum = (sum0 + sum1) + (sum2 + sum3);
@@ -457,6 +508,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         __syncwarp();
         nm_tc_fence_after();
         nm_tmem_dealloc(tmem_base, TMEM_COLS);
+        if constexpr (PT) nm_tmem_dealloc(tmem_p, P_COLS);
     }
 }
 
@@ -536,8 +588,9 @@ nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStr
     if (!nm_attention_stream_supported(d)) return NM_ERR_UNSUPPORTED;
     // the softmax input is never positive: a table whose range reaches 0 needs no upper clamp
     const bool clamp_hi = ctx->h_tables[d->exp_slot].x_max < 0.0f;
-    // one group per CTA (three CTAs per SM) measures a few percent faster up to L = 512, two groups beyond
-    const int groups = ctx->attn_groups ? ctx->attn_groups : (d->L <= 512 ? 1 : 2);
+    // one group per CTA (three CTAs per SM, P through tensor memory) measures faster at every length tried
+    // (L = 128 ... 2048: 10 % at 512 and 2048); the two-group form stays selectable for comparison
+    const int groups = ctx->attn_groups ? ctx->attn_groups : 1;
     if (groups == 1) {
         if (d->dtype == NM_BF16)
             return clamp_hi ? launch<__nv_bfloat16, true, 1>(ctx, d, st, out_q, q_inv_scale) : launch<__nv_bfloat16, false, 1>(ctx, d, st, out_q, q_inv_scale);
