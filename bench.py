@@ -50,6 +50,8 @@ def parse_args():
     p.add_argument("--no-rows-leg", action="store_true",
                    help="encoder workloads: skip the row-kernel bandwidth leg on a tensor beyond L2")
     p.add_argument("--repeats", type=int, default=REPEATS, help="how many times the K-step timed region is run")
+    p.add_argument("--streams", type=int, default=2, choices=[1, 2],
+                   help="steps in flight: 2 = the K steps alternate between two streams with their own buffers")
     p.add_argument("--algo", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     return p.parse_args()
 
@@ -144,6 +146,32 @@ def physical_gpu_index(local):
 # workloads
 # ----------------------------------------------------------------------------------------------
 
+def fork_streams(wl, stream):
+    """Two slots (device input, device output, workspace, pinned result, stream) for steps in flight together;
+    slot 0 is the workload's own buffers.  Both streams are ordered after what `stream` holds."""
+    import torch
+    if not hasattr(wl, "slots"):
+        ws = wl.model.workspace
+        x2 = wl.x.clone()
+        wl.slots = [(wl.x, wl.y, ws, wl.yh, torch.cuda.Stream()),
+                    (x2, torch.empty_like(wl.y), torch.empty_like(ws), torch.empty_like(wl.yh).pin_memory(),
+                     torch.cuda.Stream())]
+        torch.cuda.synchronize()
+    start = torch.cuda.Event()
+    start.record(stream)
+    for sl in wl.slots:
+        sl[4].wait_event(start)
+
+
+def join_streams(wl, stream):
+    """`stream` waits for everything the two slot streams hold."""
+    import torch
+    for sl in wl.slots:
+        done = torch.cuda.Event()
+        done.record(sl[4])
+        stream.wait_event(done)
+
+
 class EncoderWorkload:
     """c1..c4: the PWL transformer encoder stack; unit = tokens."""
     metric = "PWL BERT encoder tokens/s"
@@ -198,6 +226,29 @@ class EncoderWorkload:
     def host_step(self):
         m = self.model
         self.ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, self.xh, self.yh, self.x, self.y, m.workspace)
+
+    e2e_pipeline = "2 streams, each with its own device buffers, workspace and pinned result buffer"
+
+    def host_steps(self, k, stream):
+        """k calls of nm_encoder_stack_host_async, alternating between two streams: the copies of one call
+        overlap the kernels of the other.  Everything is ordered after what `stream` holds, and `stream`
+        waits for both at the end."""
+        m = self.model
+        fork_streams(self, stream)
+        for i in range(k):
+            x, y, ws, yh, st = self.slots[i % 2]
+            self.ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, self.xh, yh, x, y, ws, stream=st, wait=False)
+        join_streams(self, stream)
+
+    def device_steps(self, k, stream):
+        """k steps on device-resident inputs, alternating between the two streams (independent batches: the
+        ramp and drain of one step's kernels overlap the other's)."""
+        m = self.model
+        fork_streams(self, stream)
+        for i in range(k):
+            x, y, ws, yh, st = self.slots[i % 2]
+            self.ctx.encoder_stack(m.array, m.n_layers, m.ccfg, x, y, ws, stream=st)
+        join_streams(self, stream)
 
     # -- the oracle, as it stands, on whole sampled sequences (sequences are independent) -----------
     def _oracle_tables(self):
@@ -314,6 +365,26 @@ class ResnetWorkload:
     def host_step(self):
         m = self.model
         self.ctx.resnet50_forward_host(m.array, m.fc_w, m.fc_b, m.cfg, self.xh, self.yh, self.x, self.y, m.workspace)
+
+    e2e_pipeline = "2 streams, each with its own device buffers, workspace and pinned result buffer"
+
+    def host_steps(self, k, stream):
+        """k calls of nm_resnet50_forward_host_async, alternating between two streams."""
+        m = self.model
+        fork_streams(self, stream)
+        for i in range(k):
+            x, y, ws, yh, st = self.slots[i % 2]
+            self.ctx.resnet50_forward_host(m.array, m.fc_w, m.fc_b, m.cfg, self.xh, yh, x, y, ws, stream=st, wait=False)
+        join_streams(self, stream)
+
+    def device_steps(self, k, stream):
+        """k steps on device-resident inputs, alternating between the two streams."""
+        m = self.model
+        fork_streams(self, stream)
+        for i in range(k):
+            x, y, ws, yh, st = self.slots[i % 2]
+            self.ctx.resnet50_forward(m.array, m.fc_w, m.fc_b, m.cfg, x, y, ws, stream=st)
+        join_streams(self, stream)
 
     def _oracle_run(self, n_img):
         import oracle
@@ -573,6 +644,10 @@ def main():
     warm = max(args.warmup, 3)
     for _ in range(warm):
         wl.step()
+    two_streams = args.streams == 2 and hasattr(wl, "device_steps")
+    if two_streams:
+        wl.device_steps(4, stream)   # allocates the second slot and warms both streams
+        torch.cuda.synchronize()
     ctx.check_device_status()
 
     # ---- timed region: K steps between two CUDA events on the launching stream, barrier and synchronize
@@ -588,12 +663,24 @@ def main():
         ctx.launch_count(reset=True)
         barrier()
         ev0.record(stream)
-        for _ in range(args.steps):
-            wl.step()
+        if two_streams:
+            wl.device_steps(args.steps, stream)
+        else:
+            for _ in range(args.steps):
+                wl.step()
         ev1.record(stream)
         barrier()
         reps.append(max_over_ranks(ev0.elapsed_time(ev1)) / args.steps)
         launches = ctx.launch_count()
+    single_ms = None
+    if two_streams:   # the same K steps one after another on one stream, once, for comparison
+        barrier()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            wl.step()
+        ev1.record(stream)
+        barrier()
+        single_ms = max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
     sampler.stop()
     ctx.check_device_status()
     srt = sorted(reps)
@@ -615,7 +702,11 @@ def main():
     ctx.profile_enable(False)
 
     # ---- end to end through the C ABI with host buffers ------------------------------------
-    e2e_steps = max(3, min(args.steps, 20))
+    # Every step copies its input from pinned host memory and its result back, inside the timed region.  The
+    # encoder and CNN workloads issue the steps through the library's asynchronous host-buffer call on two
+    # streams, so that one step's copies overlap the other's kernels (reported under "pipeline"); the same
+    # loop with the blocking call, one step at a time, is reported as "serial_ms_per_step".
+    e2e_steps = max(4, min(args.steps, 20))
     wl.host_step()
     barrier()
     e0 = torch.cuda.Event(enable_timing=True)
@@ -625,7 +716,16 @@ def main():
         wl.host_step()
     e1.record(stream)
     barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    e2e_serial_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    e2e_ms = e2e_serial_ms
+    if hasattr(wl, "host_steps"):
+        wl.host_steps(2, stream)   # allocates the second slot, warms both streams
+        barrier()
+        e0.record(stream)
+        wl.host_steps(e2e_steps, stream)
+        e1.record(stream)
+        barrier()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
 
     if rank == 0:
         peaks, peak_kind = load_peaks()
@@ -670,12 +770,19 @@ def main():
         line = {
             "metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config(world),
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": dict(wl.config(world), streams=2 if two_streams else 1),
+            "streams": {"n": 2 if two_streams else 1, "single_stream_ms_per_step": single_ms,
+                        "note": "the K timed steps alternate between two CUDA streams, each with its own input, "
+                                "output and workspace (independent batches in flight together)" if two_streams
+                                else "one step after another on one stream"},
             "repeats": {"n": len(reps), "ms_per_step": [round(r, 5) for r in reps], "min": srt[0], "max": srt[-1],
                         "spread": (srt[-1] - srt[0]) / ms_step, "value_is": "median"},
             "clocks": clocks,
             "e2e": {"value": world * getattr(wl, "e2e_units", wl.units_per_step) / (e2e_ms * 1e-3), "unit": wl.unit,
-                    "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": e2e_ms},
+                    "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": e2e_ms,
+                    "serial_ms_per_step": e2e_serial_ms,
+                    "pipeline": getattr(wl, "e2e_pipeline", "none: one blocking call per step")},
             "gpu_launches": launches,
             "roofline": roofline,
             "roofline_other": extra,

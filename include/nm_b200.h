@@ -304,6 +304,14 @@ nm_status nm_encoder_stack(nm_ctx* ctx, const nm_encoder_weights* layers, int32_
 nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, int32_t n_layers,
                                 const nm_encoder_cfg* cfg, const void* x_host, void* y_host,
                                 void* x_dev, void* y_dev, void* workspace, size_t ws_bytes, void* stream);
+/* The same without the final wait: the two copies and the kernels are only enqueued on `stream`; y_host
+ * holds the result once the caller has synchronised that stream (or an event recorded after the call).
+ * x_host and y_host should be page-locked so that the copies run asynchronously.  Calls on different
+ * streams, each with its own x_dev, y_dev and workspace, may be in flight together (their copies then
+ * overlap the other call's kernels); the tables of `ctx` must not be reloaded meanwhile. */
+nm_status nm_encoder_stack_host_async(nm_ctx* ctx, const nm_encoder_weights* layers, int32_t n_layers,
+                                      const nm_encoder_cfg* cfg, const void* x_host, void* y_host,
+                                      void* x_dev, void* y_dev, void* workspace, size_t ws_bytes, void* stream);
 
 /* 2-D convolution with PWL epilogue, NHWC (Section 3.1: convolution kernels are linear
  * operations whose matrix dimensions follow from width, height and channels; Section 3: ReLU
@@ -384,6 +392,11 @@ nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const vo
 nm_status nm_resnet50_forward_host(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w, const float* fc_b,
                                    const nm_resnet50_cfg* cfg, const void* x_host, void* logits_host, void* x_dev,
                                    void* logits_dev, void* workspace, size_t ws_bytes, void* stream);
+/* The same without the final wait (see nm_encoder_stack_host_async). */
+nm_status nm_resnet50_forward_host_async(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w,
+                                         const float* fc_b, const nm_resnet50_cfg* cfg, const void* x_host,
+                                         void* logits_host, void* x_dev, void* logits_dev, void* workspace,
+                                         size_t ws_bytes, void* stream);
 
 /* nm_encoder_layer for callers that cannot provide a workspace.  (The paper has no
  * counterpart to this call: it exists for the library's users, not for the method.)

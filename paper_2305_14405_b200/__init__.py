@@ -30,7 +30,7 @@ EXPORTS = [
     "nm_encoder_stack_host", "nm_ctx_profile_enable", "nm_ctx_profile_read", "nm_encoder_layer_static",
     "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_maxpool2d_pwl", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
     "nm_resnet50_forward", "nm_resnet50_forward_host", "nm_pwl_table_build_elastic",
-    "nm_selftest_bounded_wait", "nm_attention_pwl_i8",
+    "nm_selftest_bounded_wait", "nm_attention_pwl_i8", "nm_encoder_stack_host_async", "nm_resnet50_forward_host_async",
 ]
 KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc",
                 "im2col", "pool")
@@ -142,6 +142,7 @@ def load():
     lib.nm_encoder_stack_host.argtypes = [C.c_void_p, C.POINTER(EncoderWeights), C.c_int32, C.POINTER(EncoderCfg),
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                           C.c_void_p]
+    lib.nm_encoder_stack_host_async.argtypes = lib.nm_encoder_stack_host.argtypes
     lib.nm_encoder_layer_static.argtypes = [C.c_void_p, C.POINTER(EncoderWeights), C.POINTER(EncoderCfg), C.c_void_p,
                                             C.c_void_p, C.c_void_p]
     lib.nm_conv2d_workspace_bytes.restype = C.c_size_t
@@ -158,6 +159,7 @@ def load():
     lib.nm_resnet50_forward_host.argtypes = [C.c_void_p, C.POINTER(ConvParams), C.c_void_p, C.c_void_p,
                                              C.POINTER(Resnet50Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.nm_resnet50_forward_host_async.argtypes = lib.nm_resnet50_forward_host.argtypes
     lib.nm_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.nm_ctx_profile_enable.argtypes = [C.c_void_p, C.c_int]
     lib.nm_ctx_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_double),
@@ -417,12 +419,13 @@ class Context:
                "nm_resnet50_forward")
 
     def resnet50_forward_host(self, conv_array, fc_w, fc_b, cfg, x_host, logits_host, x_dev, logits_dev, workspace,
-                              stream=None):
-        _check(self._lib.nm_resnet50_forward_host(self._h, conv_array, _ptr(fc_w), _ptr(fc_b), C.byref(cfg),
-                                                  C.c_void_p(x_host.data_ptr()), C.c_void_p(logits_host.data_ptr()),
-                                                  _ptr(x_dev), _ptr(logits_dev), _ptr(workspace),
-                                                  workspace.numel() * workspace.element_size(), _stream(stream)),
-               "nm_resnet50_forward_host")
+                              stream=None, wait=True):
+        """wait=False: nm_resnet50_forward_host_async (the caller synchronises the stream)."""
+        name = "nm_resnet50_forward_host" if wait else "nm_resnet50_forward_host_async"
+        _check(getattr(self._lib, name)(self._h, conv_array, _ptr(fc_w), _ptr(fc_b), C.byref(cfg),
+                                        C.c_void_p(x_host.data_ptr()), C.c_void_p(logits_host.data_ptr()),
+                                        _ptr(x_dev), _ptr(logits_dev), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream)), name)
 
     # -- encoder ------------------------------------------------------------------
     @staticmethod
@@ -467,13 +470,15 @@ class Context:
                                           _ptr(workspace), workspace.numel() * workspace.element_size(),
                                           _stream(stream)), "nm_encoder_stack")
 
-    def encoder_stack_host(self, layer_array, n_layers, cfg, x_host, y_host, x_dev, y_dev, workspace, stream=None):
-        """x_host / y_host: CPU tensors (pinned for full copy speed)."""
-        _check(self._lib.nm_encoder_stack_host(self._h, layer_array, n_layers, C.byref(cfg),
-                                               C.c_void_p(x_host.data_ptr()), C.c_void_p(y_host.data_ptr()),
-                                               _ptr(x_dev), _ptr(y_dev), _ptr(workspace),
-                                               workspace.numel() * workspace.element_size(), _stream(stream)),
-               "nm_encoder_stack_host")
+    def encoder_stack_host(self, layer_array, n_layers, cfg, x_host, y_host, x_dev, y_dev, workspace, stream=None,
+                           wait=True):
+        """x_host / y_host: CPU tensors (pinned for full copy speed).  wait=False: nm_encoder_stack_host_async
+        (the caller synchronises the stream before reading y_host)."""
+        name = "nm_encoder_stack_host" if wait else "nm_encoder_stack_host_async"
+        _check(getattr(self._lib, name)(self._h, layer_array, n_layers, C.byref(cfg),
+                                        C.c_void_p(x_host.data_ptr()), C.c_void_p(y_host.data_ptr()),
+                                        _ptr(x_dev), _ptr(y_dev), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream)), name)
 
 
 def layer_array(weight_structs):

@@ -335,9 +335,10 @@ nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const vo
     return nm_linear_pwl(ctx, &ld, stream);
 }
 
-nm_status nm_resnet50_forward_host(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w, const float* fc_b,
-                                   const nm_resnet50_cfg* cfg, const void* x_host, void* logits_host, void* x_dev,
-                                   void* logits_dev, void* workspace, size_t ws_bytes, void* stream)
+nm_status nm_resnet50_forward_host_async(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w,
+                                         const float* fc_b, const nm_resnet50_cfg* cfg, const void* x_host,
+                                         void* logits_host, void* x_dev, void* logits_dev, void* workspace,
+                                         size_t ws_bytes, void* stream)
 {
     if (!ctx || !cfg || !x_host || !logits_host || !x_dev || !logits_dev) return NM_ERR_INVALID_ARG;
     if (cfg->batch < 1 || cfg->num_classes < 1) return NM_ERR_SHAPE;
@@ -347,7 +348,17 @@ nm_status nm_resnet50_forward_host(nm_ctx* ctx, const nm_conv_params* convs, con
     nm_status s = nm_resnet50_forward(ctx, convs, fc_w, fc_b, cfg, x_dev, logits_dev, workspace, ws_bytes, stream);
     if (s != NM_OK) return s;
     NM_CUDA_TRY(cudaMemcpyAsync(logits_host, logits_dev, lb, cudaMemcpyDeviceToHost, st));
-    NM_CUDA_TRY(cudaStreamSynchronize(st));
+    return NM_OK;
+}
+
+nm_status nm_resnet50_forward_host(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w, const float* fc_b,
+                                   const nm_resnet50_cfg* cfg, const void* x_host, void* logits_host, void* x_dev,
+                                   void* logits_dev, void* workspace, size_t ws_bytes, void* stream)
+{
+    nm_status s = nm_resnet50_forward_host_async(ctx, convs, fc_w, fc_b, cfg, x_host, logits_host, x_dev, logits_dev,
+                                                 workspace, ws_bytes, stream);
+    if (s != NM_OK) return s;
+    NM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return NM_OK;
 }
 

@@ -632,9 +632,9 @@ nm_status nm_encoder_stack(nm_ctx* ctx, const nm_encoder_weights* layers, int32_
     return NM_OK;
 }
 
-nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, int32_t n_layers,
-                                const nm_encoder_cfg* c, const void* x_host, void* y_host, void* x_dev, void* y_dev,
-                                void* workspace, size_t ws_bytes, void* stream)
+nm_status nm_encoder_stack_host_async(nm_ctx* ctx, const nm_encoder_weights* layers, int32_t n_layers,
+                                      const nm_encoder_cfg* c, const void* x_host, void* y_host, void* x_dev,
+                                      void* y_dev, void* workspace, size_t ws_bytes, void* stream)
 {
     if (!ctx || !c || !x_host || !y_host || !x_dev || !y_dev) return NM_ERR_INVALID_ARG;
     if (c->B < 1 || c->L < 1 || c->H < 1) return NM_ERR_SHAPE;
@@ -644,7 +644,17 @@ nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, i
     nm_status s = nm_encoder_stack(ctx, layers, n_layers, c, x_dev, y_dev, workspace, ws_bytes, stream);
     if (s != NM_OK) return s;
     NM_CUDA_TRY(cudaMemcpyAsync(y_host, y_dev, bytes, cudaMemcpyDeviceToHost, st));
-    NM_CUDA_TRY(cudaStreamSynchronize(st));
+    return NM_OK;
+}
+
+nm_status nm_encoder_stack_host(nm_ctx* ctx, const nm_encoder_weights* layers, int32_t n_layers,
+                                const nm_encoder_cfg* c, const void* x_host, void* y_host, void* x_dev, void* y_dev,
+                                void* workspace, size_t ws_bytes, void* stream)
+{
+    nm_status s = nm_encoder_stack_host_async(ctx, layers, n_layers, c, x_host, y_host, x_dev, y_dev, workspace,
+                                              ws_bytes, stream);
+    if (s != NM_OK) return s;
+    NM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return NM_OK;
 }
 

@@ -135,6 +135,36 @@ def test_encoder_host_entry_point(nm, ctx):
     assert torch.equal(yh, y.cpu())
 
 
+def test_encoder_host_entry_point_async_two_streams(nm, ctx):
+    """Six asynchronous host-buffer calls alternating between two streams, each with its own device buffers and
+    workspace, different inputs per call: every result equals the blocking call's."""
+    cfg = nm_inputs.with_(nm_inputs.C2, B=2)
+    load_tables_both(ctx, cfg.segments, cfg.ranges())
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=1, layers=2)
+    m = build(nm, ctx, cfg, layers)
+    base = torch.from_numpy(x).bfloat16()
+    xs = [(base * (1.0 + 0.05 * i)).pin_memory() for i in range(6)]
+    want = []
+    xd = torch.empty(base.shape, dtype=torch.bfloat16, device="cuda")
+    yd = torch.empty_like(xd)
+    for xh in xs:
+        yh = torch.empty_like(xh).pin_memory()
+        ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, xh, yh, xd, yd, m.workspace)
+        want.append(yh.clone())
+    slots = [(torch.empty_like(xd), torch.empty_like(yd), torch.empty_like(m.workspace), torch.cuda.Stream())
+             for _ in range(2)]
+    outs = [torch.empty_like(xs[0]).pin_memory() for _ in range(6)]
+    torch.cuda.synchronize()
+    for i, xh in enumerate(xs):
+        sx, sy, ws, st = slots[i % 2]
+        ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, xh, outs[i], sx, sy, ws, stream=st, wait=False)
+    torch.cuda.synchronize()
+    ctx.check_device_status()
+    for i in range(6):
+        assert torch.equal(outs[i], want[i]), i
+    assert not torch.equal(want[0], want[1])
+
+
 def test_encoder_workspace_errors(nm, ctx):
     cfg = nm_inputs.with_(nm_inputs.C2, B=1)
     load_tables_both(ctx, cfg.segments, cfg.ranges())
