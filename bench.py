@@ -50,8 +50,8 @@ def parse_args():
     p.add_argument("--no-rows-leg", action="store_true",
                    help="encoder workloads: skip the row-kernel bandwidth leg on a tensor beyond L2")
     p.add_argument("--repeats", type=int, default=REPEATS, help="how many times the K-step timed region is run")
-    p.add_argument("--streams", type=int, default=2, choices=[1, 2],
-                   help="steps in flight: 2 = the K steps alternate between two streams with their own buffers")
+    p.add_argument("--streams", type=int, default=2, choices=[1, 2, 3, 4],
+                   help="steps in flight: n > 1 = the K steps rotate over n streams, each with its own buffers")
     p.add_argument("--algo", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     return p.parse_args()
 
@@ -152,10 +152,10 @@ def fork_streams(wl, stream):
     import torch
     if not hasattr(wl, "slots"):
         ws = wl.model.workspace
-        x2 = wl.x.clone()
-        wl.slots = [(wl.x, wl.y, ws, wl.yh, torch.cuda.Stream()),
-                    (x2, torch.empty_like(wl.y), torch.empty_like(ws), torch.empty_like(wl.yh).pin_memory(),
-                     torch.cuda.Stream())]
+        wl.slots = [(wl.x, wl.y, ws, wl.yh, torch.cuda.Stream())]
+        for _ in range(1, max(2, wl.args.streams)):
+            wl.slots.append((wl.x.clone(), torch.empty_like(wl.y), torch.empty_like(ws),
+                             torch.empty_like(wl.yh).pin_memory(), torch.cuda.Stream()))
         torch.cuda.synchronize()
     start = torch.cuda.Event()
     start.record(stream)
@@ -227,7 +227,7 @@ class EncoderWorkload:
         m = self.model
         self.ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, self.xh, self.yh, self.x, self.y, m.workspace)
 
-    e2e_pipeline = "2 streams, each with its own device buffers, workspace and pinned result buffer"
+    e2e_pipeline = "one stream per step in flight (--streams), each with its own device buffers, workspace and pinned result buffer"
 
     def host_steps(self, k, stream):
         """k calls of nm_encoder_stack_host_async, alternating between two streams: the copies of one call
@@ -236,7 +236,7 @@ class EncoderWorkload:
         m = self.model
         fork_streams(self, stream)
         for i in range(k):
-            x, y, ws, yh, st = self.slots[i % 2]
+            x, y, ws, yh, st = self.slots[i % len(self.slots)]
             self.ctx.encoder_stack_host(m.array, m.n_layers, m.ccfg, self.xh, yh, x, y, ws, stream=st, wait=False)
         join_streams(self, stream)
 
@@ -246,7 +246,7 @@ class EncoderWorkload:
         m = self.model
         fork_streams(self, stream)
         for i in range(k):
-            x, y, ws, yh, st = self.slots[i % 2]
+            x, y, ws, yh, st = self.slots[i % len(self.slots)]
             self.ctx.encoder_stack(m.array, m.n_layers, m.ccfg, x, y, ws, stream=st)
         join_streams(self, stream)
 
@@ -366,14 +366,14 @@ class ResnetWorkload:
         m = self.model
         self.ctx.resnet50_forward_host(m.array, m.fc_w, m.fc_b, m.cfg, self.xh, self.yh, self.x, self.y, m.workspace)
 
-    e2e_pipeline = "2 streams, each with its own device buffers, workspace and pinned result buffer"
+    e2e_pipeline = "one stream per step in flight (--streams), each with its own device buffers, workspace and pinned result buffer"
 
     def host_steps(self, k, stream):
         """k calls of nm_resnet50_forward_host_async, alternating between two streams."""
         m = self.model
         fork_streams(self, stream)
         for i in range(k):
-            x, y, ws, yh, st = self.slots[i % 2]
+            x, y, ws, yh, st = self.slots[i % len(self.slots)]
             self.ctx.resnet50_forward_host(m.array, m.fc_w, m.fc_b, m.cfg, self.xh, yh, x, y, ws, stream=st, wait=False)
         join_streams(self, stream)
 
@@ -382,7 +382,7 @@ class ResnetWorkload:
         m = self.model
         fork_streams(self, stream)
         for i in range(k):
-            x, y, ws, yh, st = self.slots[i % 2]
+            x, y, ws, yh, st = self.slots[i % len(self.slots)]
             self.ctx.resnet50_forward(m.array, m.fc_w, m.fc_b, m.cfg, x, y, ws, stream=st)
         join_streams(self, stream)
 
@@ -644,7 +644,7 @@ def main():
     warm = max(args.warmup, 3)
     for _ in range(warm):
         wl.step()
-    two_streams = args.streams == 2 and hasattr(wl, "device_steps")
+    two_streams = args.streams >= 2 and hasattr(wl, "device_steps")
     if two_streams:
         wl.device_steps(4, stream)   # allocates the second slot and warms both streams
         torch.cuda.synchronize()
@@ -771,9 +771,9 @@ def main():
             "metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-            "config": dict(wl.config(world), streams=2 if two_streams else 1),
-            "streams": {"n": 2 if two_streams else 1, "single_stream_ms_per_step": single_ms,
-                        "note": "the K timed steps alternate between two CUDA streams, each with its own input, "
+            "config": dict(wl.config(world), streams=args.streams if two_streams else 1),
+            "streams": {"n": args.streams if two_streams else 1, "single_stream_ms_per_step": single_ms,
+                        "note": "the K timed steps rotate over the CUDA streams, each with its own input, "
                                 "output and workspace (independent batches in flight together)" if two_streams
                                 else "one step after another on one stream"},
             "repeats": {"n": len(reps), "ms_per_step": [round(r, 5) for r in reps], "min": srt[0], "max": srt[-1],
