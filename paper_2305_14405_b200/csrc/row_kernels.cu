@@ -75,8 +75,11 @@ __global__ void __launch_bounds__(256) pwl_apply_kernel(const NmTable* __restric
 
 // ---- LayerNorm with PWL rsqrt: one warp per row, the row kept in registers ------
 //   mu = mean(z); v = mean((z-mu)^2); r = PWL_rsqrt(v + eps); y = (z-mu)*r*gamma + beta
-template <typename T, int ITERS>
-__global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restrict__ tab,
+// GB_REGS: the lane's gamma and beta values stay in registers for all of the warp's rows (2 x ITERS x N
+// registers: rows up to 32 x 3 vectors, two blocks per SM).  Otherwise they are fetched per row through L1,
+// which then carries four times the bytes of the row itself and ~700 exposed cycles per row.
+template <typename T, int ITERS, bool GB_REGS>
+__global__ void __launch_bounds__(256, GB_REGS ? 2 : 1) layernorm_kernel(const NmTable* __restrict__ tab,
                                                         const NmTable* __restrict__ tab2, const T* __restrict__ x,
                                                         const float* __restrict__ gamma,
                                                         const float* __restrict__ beta, T* __restrict__ y,
@@ -100,6 +103,20 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restric
         for (int it = 0; it < ITERS; ++it) {
             const int v = it * 32 + lane;
             if (v < nvec) nxt[it] = *reinterpret_cast<const uint4*>(x + warp0 * H + v * N);
+        }
+    }
+    float rg[GB_REGS ? ITERS : 1][N], rb[GB_REGS ? ITERS : 1][N];
+    if constexpr (GB_REGS) {
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            const int v = it * 32 + lane;
+            if (v < nvec) {
+#pragma unroll
+                for (int i = 0; i < N; i += 4) {
+                    *reinterpret_cast<float4*>(&rg[it][i]) = __ldg(reinterpret_cast<const float4*>(gamma + v * N + i));
+                    *reinterpret_cast<float4*>(&rb[it][i]) = __ldg(reinterpret_cast<const float4*>(beta + v * N + i));
+                }
+            }
         }
     }
     for (int64_t row = warp0; row < rows; row += nwarps) {
@@ -158,10 +175,18 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const NmTable* __restric
             const int v = it * 32 + lane;
             if (v < nvec) {
                 float g[N], b[N];
+                if constexpr (GB_REGS) {
 #pragma unroll
-                for (int i = 0; i < N; i += 4) {
-                    *reinterpret_cast<float4*>(&g[i]) = __ldg(reinterpret_cast<const float4*>(gamma + v * N + i));
-                    *reinterpret_cast<float4*>(&b[i]) = __ldg(reinterpret_cast<const float4*>(beta + v * N + i));
+                    for (int i = 0; i < N; ++i) {
+                        g[i] = rg[it][i];
+                        b[i] = rb[it][i];
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < N; i += 4) {
+                        *reinterpret_cast<float4*>(&g[i]) = __ldg(reinterpret_cast<const float4*>(gamma + v * N + i));
+                        *reinterpret_cast<float4*>(&b[i]) = __ldg(reinterpret_cast<const float4*>(beta + v * N + i));
+                    }
                 }
 #pragma unroll
                 for (int i = 0; i < N; ++i) f[it][i] = __fmaf_rn(f[it][i] * r, g[i], b[i]);
@@ -233,9 +258,12 @@ nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const NmTable* tab2, const 
     const int nvec = H / N;
     const int iters = (nvec + 31) / 32;
     const int threads = 256;
-    // a multiple of the SM count: 6 blocks of 8 warps per SM, each warp walking over rows
+    // Tensors that fit the L2 (the encoder's: 16384 x 768 is 25 MB) are latency-bound: gamma and beta in registers,
+    // one resident wave of 2 blocks per SM, 9.9 instead of 13.3 us for that shape.  Tensors far beyond the L2 are
+    // bandwidth-bound and want more warps per SM: the per-row fetch of gamma and beta, 6 blocks of 8 warps per SM
+    // (5.5 instead of 4.9 TB/s at 2^19 x 768).
+    const bool small = (double)rows * H * sizeof(T) <= 48e6 && iters <= 3;
     int64_t blocks = (rows + 7) / 8;
-    if (blocks > (int64_t)ctx->sm_count * 6) blocks = (int64_t)ctx->sm_count * 6;
  NmLaunchScope scope(ctx, NM_KERNEL_LAYERNORM, 2.0 * (double)rows * H * sizeof(T), st);
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -249,14 +277,27 @@ nm_status launch_ln(nm_ctx* ctx, const NmTable* tab, const NmTable* tab2, const 
     cfg.numAttrs = ctx->pdl ? 1 : 0;
     const T* xt = (const T*)x;
     T* yt = (T*)y;
-#define NM_LN_CASE(I) \
-    cudaLaunchKernelEx(&cfg, layernorm_kernel<T, I>, tab, tab2, xt, gamma, beta, yt, rows, H, eps, q, q_inv_scale)
-    if (iters <= 1) NM_LN_CASE(1);
-    else if (iters <= 2) NM_LN_CASE(2);
-    else if (iters <= 3) NM_LN_CASE(3);
-    else if (iters <= 4) NM_LN_CASE(4);
-    else if (iters <= 8) NM_LN_CASE(8);
-    else if (iters <= 16) NM_LN_CASE(16);
+#define NM_LN_CASE(I, GB)                                                                                     \
+    do {                                                                                                      \
+        static int resident = 0;   /* blocks per SM that this instantiation's registers allow */              \
+        if (GB && resident == 0 &&                                                                            \
+            (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, layernorm_kernel<T, I, GB>, threads, 0) != \
+                 cudaSuccess || resident < 1))                                                                \
+            resident = 2;                                                                                     \
+        const int64_t cap = (int64_t)ctx->sm_count * (GB ? resident : 6);                                     \
+        cfg.gridDim = dim3((unsigned)(blocks > cap ? cap : blocks));                                          \
+        cudaLaunchKernelEx(&cfg, layernorm_kernel<T, I, GB>, tab, tab2, xt, gamma, beta, yt, rows, H, eps, q,  \
+                           q_inv_scale);                                                                      \
+    } while (0)
+    if (small && iters <= 1) NM_LN_CASE(1, true);
+    else if (small && iters <= 2) NM_LN_CASE(2, true);
+    else if (small && iters <= 3) NM_LN_CASE(3, true);
+    else if (iters <= 1) NM_LN_CASE(1, false);
+    else if (iters <= 2) NM_LN_CASE(2, false);
+    else if (iters <= 3) NM_LN_CASE(3, false);
+    else if (iters <= 4) NM_LN_CASE(4, false);
+    else if (iters <= 8) NM_LN_CASE(8, false);
+    else if (iters <= 16) NM_LN_CASE(16, false);
     else return NM_ERR_UNSUPPORTED;
 #undef NM_LN_CASE
     return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
