@@ -109,6 +109,52 @@ __device__ __forceinline__ float max3f(float a, float b, float c)
     return d;
 }
 
+// A tile is one (batch, head, 128-query block); tile index = (b * heads + g) * blocks_per_seq + qb.
+struct Tile { int qb, g, b; };
+struct TileGeom { int blocks_per_seq, heads; };
+__device__ __forceinline__ Tile tile_decode(const TileGeom& gm, int t)
+{
+    Tile r;
+    r.qb = t % gm.blocks_per_seq;
+    r.g = (t / gm.blocks_per_seq) % gm.heads;
+    r.b = t / (gm.blocks_per_seq * gm.heads);
+    return r;
+}
+// What the first loads of a tile need: tensor maps, staging buffers, their barriers.
+struct LoadCtx {
+    const CUtensorMap *tmQ, *tmK, *tmV;
+    uint8_t *q_s, *k_st, *p_s, *v_st;
+    uint64_t *bar_q, *bar_k1_full, *bar_v_full;   // bar_k1_full: [group][2]
+    int n128;
+};
+// Q and each group's first two 128-key chunks of sweep 1 (stage 0 = the group's two K stages, stage 1 = its P
+// tile).  One thread; the buffers must be free.
+template <int NG>
+__device__ __forceinline__ void load_tile_head(const LoadCtx& c, const Tile& t)
+{
+    nm_mbar_expect_tx(c.bar_q, BQ * ROWB);
+    nm_tma_load_3d(c.q_s, c.tmQ, t.g * HD, t.qb * BQ, t.b, c.bar_q);
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+#pragma unroll
+        for (int st = 0; st < 2; ++st) {
+            const int c128 = gi + NG * st;
+            if (c128 >= c.n128) break;
+            uint8_t* dst = st == 0 ? c.k_st + (size_t)gi * 2 * STAGE : c.p_s + (size_t)gi * PBUF;
+            uint64_t* bar = c.bar_k1_full + gi * 2 + st;
+            nm_mbar_expect_tx(bar, 2 * STAGE);
+            nm_tma_load_3d(dst, c.tmK, t.g * HD, c128 * 2 * CK, t.b, bar);
+            nm_tma_load_3d(dst + STAGE, c.tmK, t.g * HD, c128 * 2 * CK + CK, t.b, bar);
+        }
+    }
+}
+// The group's first V chunk of a tile (one thread; the V stage must be free).
+__device__ __forceinline__ void load_first_v(const LoadCtx& c, const Tile& t, int gi)
+{
+    nm_mbar_expect_tx(c.bar_v_full + gi, STAGE);
+    nm_tma_load_3d(c.v_st + (size_t)gi * STAGE, c.tmV, t.g * HD, gi * CK, t.b, c.bar_v_full + gi);
+}
+
 // NG = softmax groups per CTA: 2 (320 threads, 256 tensor-memory columns, two CTAs per SM) or
 // 1 (160 threads, 128 columns, three CTAs per SM: more tiles in flight per SM, fewer warps per tile).
 template <typename T, bool CLAMP_HI, int NG>
@@ -149,10 +195,18 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     float2* rep = reinterpret_cast<float2*>(p_s + NG * PBUF);   // (n_exp + 1) x 16 copies
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // A CTA walks over the (batch, head, 128-query block) tiles blockIdx.x, blockIdx.x + gridDim.x, ...: barriers,
+    // tensor memory and the replicated table are set up once, and the control warp fetches the next tile's Q,
+    // first K chunks and first V chunk while the softmax warps finish the current one.
     const int blocks_per_seq = L / BQ;
-    const int qb = blockIdx.x % blocks_per_seq;
-    const int g = (blockIdx.x / blocks_per_seq) % a.heads;
-    const int b = blockIdx.x / (blocks_per_seq * a.heads);
+    const int n_tiles = a.B * a.heads * blocks_per_seq;
+    const TileGeom geom = {blocks_per_seq, a.heads};
+    auto tile_of = [geom](int t) { return tile_decode(geom, t); };
+    LoadCtx lc;
+    lc.tmQ = &tmQ; lc.tmK = &tmK; lc.tmV = &tmV;
+    lc.q_s = q_s; lc.k_st = k_st; lc.p_s = p_s; lc.v_st = v_st;
+    lc.bar_q = &bar_q; lc.bar_k1_full = &bar_k1_full[0][0]; lc.bar_v_full = &bar_v_full[0];
+    lc.n128 = n128;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -176,19 +230,10 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         // 128-key chunks of sweep 1 (stage 0 = the group's two K stages, stage 1 = its P tile, which
         // sweep 1 does not use otherwise) and its first V chunk.
         nm_grid_dependency_wait();   // Q, K, V come from the previous kernel
-        nm_mbar_expect_tx(&bar_q, BQ * ROWB);
-        nm_tma_load_3d(q_s, &tmQ, g * HD, qb * BQ, b, &bar_q);
-        for (int gi = 0; gi < NG; ++gi) {
-            for (int st = 0; st < 2; ++st) {
-                const int c128 = gi + NG * st;
-                if (c128 >= n128) break;
-                uint8_t* dst = st == 0 ? k_st + (size_t)gi * 2 * STAGE : p_s + (size_t)gi * PBUF;
-                nm_mbar_expect_tx(&bar_k1_full[gi][st], 2 * STAGE);
-                nm_tma_load_3d(dst, &tmK, g * HD, c128 * 2 * CK, b, &bar_k1_full[gi][st]);
-                nm_tma_load_3d(dst + STAGE, &tmK, g * HD, c128 * 2 * CK + CK, b, &bar_k1_full[gi][st]);
-            }
-            nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
-            nm_tma_load_3d(v_st + (size_t)gi * STAGE, &tmV, g * HD, gi * CK, b, &bar_v_full[gi]);
+        if ((int)blockIdx.x < n_tiles) {
+            const Tile t0 = tile_of((int)blockIdx.x);
+            load_tile_head<NG>(lc, t0);
+            for (int gi = 0; gi < NG; ++gi) load_first_v(lc, t0, gi);
         }
     }
     if (warp == NG - 1) {
@@ -221,7 +266,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         //                  after next into it) and S is free (issue Q K^T for the next chunk);
         //   P-ready(j):    the bf16 P tile of the j-th chunk of sweep 2 is in shared memory -> O += P V.
         const int gi = NG == 1 ? 0 : warp;
-        const uint32_t bar_sc = 2 + 2 * gi, bar_pr = 3 + 2 * gi;
+        const uint32_t bar_sc = 2 + 2 * gi, bar_pr = 3 + 2 * gi, bar_oc = 6 + gi;
         const int cnt1 = (n128 - gi + NG - 1) / NG;   // the group's 128-key chunks in sweep 1
         uint8_t* my_k = k_st + (size_t)gi * 2 * STAGE;
         uint8_t* my_v = v_st + (size_t)gi * STAGE;
@@ -230,86 +275,117 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         auto wait = [&](uint64_t* bar, uint32_t parity) {
             return __all_sync(0xffffffffu, nm_mbar_wait_relaxed<20>(bar, parity, abortp, a.status)) != 0;
         };
-        bool ok = wait(&bar_q, 0);
+        bool ok = true;
         const uint64_t qdesc = nm_smem_desc_sw128(nm_smem_u32(q_s));
-        // ---- sweep 1: [S_g | O_g] = Q K^T for 128 keys at a time; K stage i & 1 (0: the two K stages
-        // taken together, 1: the P tile)
-        auto issue_qk1 = [&](int i) {
-            if (!ok) return;
-            if (!wait(&bar_k1_full[gi][i & 1], (uint32_t)((i >> 1) & 1))) { ok = false; return; }
-            nm_tc_fence_after();
-            const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32((i & 1) ? my_p : my_k));
-            if (nm_elect_one()) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) nm_mma_f16(my_tmem, qdesc + 2 * k, kdesc + 2 * k, IDESC_QK1, k != 0);
-                nm_tc_commit(&bar_s_full[gi]);
-            }
-            __syncwarp();
-        };
-        if (cnt1 > 0) issue_qk1(0);
-        for (int i = 0; i < cnt1; ++i) {
-            asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed: chunk i is in registers
-            if (i + 1 < cnt1) issue_qk1(i + 1);
-            if (ok && i + 2 < cnt1 && nm_elect_one()) {   // its MMAs are complete: the stage takes the chunk after next
-                uint8_t* dst = (i & 1) ? my_p : my_k;
-                const int key0 = (gi + NG * (i + 2)) * 2 * CK;
-                nm_mbar_expect_tx(&bar_k1_full[gi][i & 1], 2 * STAGE);
-                nm_tma_load_3d(dst, &tmK, g * HD, key0, b, &bar_k1_full[gi][i & 1]);
-                nm_tma_load_3d(dst + STAGE, &tmK, g * HD, key0 + CK, b, &bar_k1_full[gi][i & 1]);
-            }
-            __syncwarp();
-        }
-        // ---- sweep 2: the group's j-th chunk is the 64 keys of chunk g + NG*j; K stage j & 1
-        auto load_k = [&](int j) {
-            if (ok && nm_elect_one()) {
-                nm_mbar_expect_tx(&bar_k_full[gi][j & 1], STAGE);
-                nm_tma_load_3d(my_k + (size_t)(j & 1) * STAGE, &tmK, g * HD, (gi + NG * j) * CK, b, &bar_k_full[gi][j & 1]);
-            }
-            __syncwarp();
-        };
-        auto issue_qk = [&](int j) {   // S_g = Q K^T
-            if (!ok) return;
-            if (!wait(&bar_k_full[gi][j & 1], (uint32_t)((j >> 1) & 1))) { ok = false; return; }
-            nm_tc_fence_after();
-            const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32(my_k + (size_t)(j & 1) * STAGE));
-            if (nm_elect_one()) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) nm_mma_f16(my_tmem, qdesc + 2 * k, kdesc + 2 * k, IDESC_QK, k != 0);
-                nm_tc_commit(&bar_s_full[gi]);
-            }
-            __syncwarp();
-        };
-        load_k(0);   // every MMA of sweep 1 has completed: the K stages are free
-        if (half > 1) load_k(1);
-        issue_qk(0);
-        for (int j = 0; j < half; ++j) {
-            asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed(j)
-            if (j + 1 < half) issue_qk(j + 1);
-            if (j + 2 < half) load_k(j + 2);
-            asm volatile("bar.sync %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");   // P-ready(j)
-            if (ok && !wait(&bar_v_full[gi], (uint32_t)(j & 1))) ok = false;
-            if (ok) {
+        // completions consumed so far on each barrier (they run on from tile to tile)
+        uint32_t q_cnt = 0, k1_cnt0 = 0, k1_cnt1 = 0, k_cnt0 = 0, k_cnt1 = 0, v_cnt = 0, pv_cnt = 0;
+        for (int tile = (int)blockIdx.x, ti = 0; tile < n_tiles; tile += (int)gridDim.x, ++ti) {
+            const Tile t = tile_of(tile);
+            const int g = t.g, b = t.b;
+            const bool more = tile + (int)gridDim.x < n_tiles;
+            if (ok && !wait(&bar_q, q_cnt & 1u)) ok = false;
+            ++q_cnt;
+            // the previous tile's epilogue has read O out of tensor memory (sweep 1 writes over [S_g | O_g])
+            if (ti > 0) asm volatile("bar.sync %0, %1;" ::"r"(bar_oc), "n"(160) : "memory");
+            // ---- sweep 1: [S_g | O_g] = Q K^T for 128 keys at a time; K stage i & 1 (0: the two K stages
+            // taken together, 1: the P tile)
+            auto issue_qk1 = [&](int i) {
+                const uint32_t par = ((i & 1) ? k1_cnt1 : k1_cnt0) & 1u;
+                if (i & 1) ++k1_cnt1; else ++k1_cnt0;
+                if (!ok) return;
+                if (!wait(&bar_k1_full[gi][i & 1], par)) { ok = false; return; }
                 nm_tc_fence_after();
-                const uint64_t pdesc = nm_smem_desc_sw128(nm_smem_u32(my_p));
-                const uint32_t v_addr = nm_smem_u32(my_v);
+                const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32((i & 1) ? my_p : my_k));
                 if (nm_elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
-                        const uint64_t vdesc = nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB));
-                        if constexpr (PT) mma_f16_a_tmem(my_tmem + O_OFF, tmem_p + (uint32_t)(8 * k), vdesc, IDESC_PV, (j | k) != 0);
-                        else nm_mma_f16(my_tmem + O_OFF, pdesc + 2 * k, vdesc, IDESC_PV, (j | k) != 0);
-                    }
-                    nm_tc_commit(&bar_p_empty[gi]);
+                    for (int k = 0; k < 4; ++k) nm_mma_f16(my_tmem, qdesc + 2 * k, kdesc + 2 * k, IDESC_QK1, k != 0);
+                    nm_tc_commit(&bar_s_full[gi]);
+                }
+                __syncwarp();
+            };
+            if (cnt1 > 0) issue_qk1(0);
+            for (int i = 0; i < cnt1; ++i) {
+                asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed: chunk i is in registers
+                if (i + 1 < cnt1) issue_qk1(i + 1);
+                if (ok && i + 2 < cnt1 && nm_elect_one()) {   // its MMAs are complete: the stage takes the chunk after next
+                    uint8_t* dst = (i & 1) ? my_p : my_k;
+                    const int key0 = (gi + NG * (i + 2)) * 2 * CK;
+                    nm_mbar_expect_tx(&bar_k1_full[gi][i & 1], 2 * STAGE);
+                    nm_tma_load_3d(dst, &tmK, g * HD, key0, b, &bar_k1_full[gi][i & 1]);
+                    nm_tma_load_3d(dst + STAGE, &tmK, g * HD, key0 + CK, b, &bar_k1_full[gi][i & 1]);
                 }
                 __syncwarp();
             }
-            if (ok && j + 1 < half) {   // the V stage is free once this P V has completed (nothing else to do until then)
-                if (!wait(&bar_p_empty[gi], (uint32_t)(j & 1))) ok = false;
+            // ---- sweep 2: the group's j-th chunk is the 64 keys of chunk g + NG*j; K stage j & 1
+            auto load_k = [&](int j) {
                 if (ok && nm_elect_one()) {
-                    nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
-                    nm_tma_load_3d(my_v, &tmV, g * HD, (gi + NG * (j + 1)) * CK, b, &bar_v_full[gi]);
+                    nm_mbar_expect_tx(&bar_k_full[gi][j & 1], STAGE);
+                    nm_tma_load_3d(my_k + (size_t)(j & 1) * STAGE, &tmK, g * HD, (gi + NG * j) * CK, b, &bar_k_full[gi][j & 1]);
                 }
                 __syncwarp();
+            };
+            auto issue_qk = [&](int j) {   // S_g = Q K^T
+                const uint32_t par = ((j & 1) ? k_cnt1 : k_cnt0) & 1u;
+                if (j & 1) ++k_cnt1; else ++k_cnt0;
+                if (!ok) return;
+                if (!wait(&bar_k_full[gi][j & 1], par)) { ok = false; return; }
+                nm_tc_fence_after();
+                const uint64_t kdesc = nm_smem_desc_sw128(nm_smem_u32(my_k + (size_t)(j & 1) * STAGE));
+                if (nm_elect_one()) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) nm_mma_f16(my_tmem, qdesc + 2 * k, kdesc + 2 * k, IDESC_QK, k != 0);
+                    nm_tc_commit(&bar_s_full[gi]);
+                }
+                __syncwarp();
+            };
+            load_k(0);   // every MMA of sweep 1 has completed: the K stages are free
+            if (half > 1) load_k(1);
+            issue_qk(0);
+            for (int j = 0; j < half; ++j) {
+                asm volatile("bar.sync %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");   // S-consumed(j)
+                if (j + 1 < half) issue_qk(j + 1);
+                if (j + 2 < half) load_k(j + 2);
+                if constexpr (NG == 1) {
+                    // Last chunk: every Q K^T of the tile has completed, so Q, the K stages and the P tile (which
+                    // only sweep 1 uses when P goes through tensor memory) take the next tile's first loads now.
+                    if (j + 1 == half && more && ok && nm_elect_one()) load_tile_head<NG>(lc, tile_of(tile + (int)gridDim.x));
+                    __syncwarp();
+                }
+                asm volatile("bar.sync %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");   // P-ready(j)
+                if (ok && !wait(&bar_v_full[gi], v_cnt & 1u)) ok = false;
+                ++v_cnt;
+                if (ok) {
+                    nm_tc_fence_after();
+                    const uint64_t pdesc = nm_smem_desc_sw128(nm_smem_u32(my_p));
+                    const uint32_t v_addr = nm_smem_u32(my_v);
+                    if (nm_elect_one()) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {   // V rows (keys) 16k..16k+15: two groups of 8 rows, 1024 bytes apart
+                            const uint64_t vdesc = nm_smem_desc_sw128(v_addr + (uint32_t)(16 * k * ROWB));
+                            if constexpr (PT) mma_f16_a_tmem(my_tmem + O_OFF, tmem_p + (uint32_t)(8 * k), vdesc, IDESC_PV, (j | k) != 0);
+                            else nm_mma_f16(my_tmem + O_OFF, pdesc + 2 * k, vdesc, IDESC_PV, (j | k) != 0);
+                        }
+                        nm_tc_commit(&bar_p_empty[gi]);
+                    }
+                    __syncwarp();
+                }
+                const uint32_t pv_par = pv_cnt & 1u;   // parity of this P V's completion
+                ++pv_cnt;
+                // the V stage is free once this P V has completed (nothing else to do until then): it takes the
+                // next chunk's V, or after the last chunk the next tile's first one
+                const bool next_v = j + 1 < half || (NG == 1 && more);
+                if (ok && next_v) {
+                    if (!wait(&bar_p_empty[gi], pv_par)) ok = false;
+                    if (ok && nm_elect_one()) {
+                        if (j + 1 < half) {
+                            nm_mbar_expect_tx(&bar_v_full[gi], STAGE);
+                            nm_tma_load_3d(my_v, &tmV, g * HD, (gi + NG * (j + 1)) * CK, b, &bar_v_full[gi]);
+                        } else {
+                            load_first_v(lc, tile_of(tile + (int)gridDim.x), gi);
+                        }
+                    }
+                    __syncwarp();
+                }
             }
         }
         if (!ok) {   // after an abort: let copies land and MMAs retire (bounded) before teardown
@@ -329,13 +405,15 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         const int q = warp & 3;
         const int g2 = NG == 1 ? 0 : (warp - NG) >> 2;
         const int row = q * 32 + lane;
-        const uint32_t bar_sc = 2 + 2 * g2, bar_pr = 3 + 2 * g2;
+        const uint32_t bar_sc = 2 + 2 * g2, bar_pr = 3 + 2 * g2, bar_oc = 6 + g2;
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g2 * GRP_COLS;
         const int cnt1 = (n128 - g2 + NG - 1) / NG;   // the group's 128-key chunks in sweep 1
         const float inv_h = a.t_exp->inv_h, off = a.t_exp->off, nm1 = (float)(a.n_exp - 1);
         // this lane's copy of the replicated table, with the constant of the index trick folded in:
         // (bits << 7) = 0xA0000000 + s*128 (mod 2^32) for bits = 0x4B400000 + s
         const uint32_t rep_lane = nm_smem_u32(rep) + (uint32_t)(lane & 15) * 8u - 0xA0000000u;
+        const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(g2 * PBUF + row * ROWB);
+        const uint32_t p_row = tmem_p + ((uint32_t)(q * 32) << 16);   // this warp's lane quarter of the P columns
         int ok = 1;
         // All lanes test the barrier; only when it is not yet complete does lane 0 poll (with sleeps).
         auto wait_all = [&](uint64_t* bar, uint32_t par) {
@@ -348,155 +426,170 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (ok) (void)nm_mbar_try_wait(bar, par);
             }
         };
-        // ---- sweep 1: the final row maximum
-        float m = -INFINITY;
+        // completions consumed so far: S products of this group, P V products of every group (the same count)
+        uint32_t s_cnt = 0, pv_base = 0;
+        for (int tile = (int)blockIdx.x; tile < n_tiles; tile += (int)gridDim.x) {
+            const Tile t = tile_of(tile);
+            const int qb = t.qb, g = t.g, b = t.b;
+            const bool more = tile + (int)gridDim.x < n_tiles;
+            // ---- sweep 1: the final row maximum
+            float m = -INFINITY;
 #pragma unroll 1
-        for (int i = 0; i < cnt1; ++i) {
-            wait_all(&bar_s_full[g2], (uint32_t)(i & 1));
-            if (ok) {
-                nm_tc_fence_after();
+            for (int i = 0; i < cnt1; ++i) {
+                wait_all(&bar_s_full[g2], s_cnt & 1u);
+                ++s_cnt;
+                if (ok) {
+                    nm_tc_fence_after();
 #pragma unroll
-                for (int hh = 0; hh < 4; ++hh) {   // 128 keys: the scores span [S_g | O_g]
+                    for (int hh = 0; hh < 4; ++hh) {   // 128 keys: the scores span [S_g | O_g]
+                        uint32_t r[32];
+                        nm_tmem_ld32_sync(t_row + (uint32_t)(hh * 32), r);
+                        if (hh == 3) {   // all of it is in registers: the control warp may overwrite S
+                            nm_tc_fence_before();
+                            asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
+                        }
+                        float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+                        for (int k = 0; k < 32; k += 4) {
+                            m0 = max3f(m0, __uint_as_float(r[k]), __uint_as_float(r[k + 1]));
+                            m1 = max3f(m1, __uint_as_float(r[k + 2]), __uint_as_float(r[k + 3]));
+                        }
+                        m = max3f(m, m0, m1);
+                    }
+                } else {
+                    asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
+                }
+            }
+            if constexpr (NG == 2) {   // the two groups saw different keys of the row
+                s_red[g2][row] = m;
+                asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+                m = fmaxf(s_red[0][row], s_red[1][row]);
+                asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+            }
+            const float neg_ms = -(m * a.scale);
+            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+            // ---- sweep 2: e = PWL_exp(s - m), row sum, P tiles
+#pragma unroll 1
+            for (int j = 0; j < half; ++j) {
+                wait_all(&bar_s_full[g2], s_cnt & 1u);
+                ++s_cnt;
+                if (ok) nm_tc_fence_after();
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
                     uint32_t r[32];
-                    nm_tmem_ld32_sync(t_row + (uint32_t)(hh * 32), r);
-                    if (hh == 3) {   // all of it is in registers: the control warp may overwrite S
+                    if (ok) {
+                        nm_tmem_ld32_sync(t_row + (uint32_t)(hh * 32), r);
+                    }
+                    if (hh == 1) {
                         nm_tc_fence_before();
                         asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
                     }
-                    float m0 = -INFINITY, m1 = -INFINITY;
+                    uint32_t pk[16];   // the half's 32 exponentials, packed to 16 bits
+                    if (ok) {
 #pragma unroll
-                    for (int k = 0; k < 32; k += 4) {
-                        m0 = max3f(m0, __uint_as_float(r[k]), __uint_as_float(r[k + 1]));
-                        m1 = max3f(m1, __uint_as_float(r[k + 2]), __uint_as_float(r[k + 3]));
+                        for (int jj = 0; jj < 4; ++jj) {   // 8 keys = one 16-byte chunk of the P row
+                            float e[8];
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const float x = __fmaf_rn(__uint_as_float(r[jj * 8 + k]), a.scale, neg_ms);
+                                float u = fmaxf(__fmaf_rn(x, inv_h, off), 0.0f);
+                                if (CLAMP_HI) u = fminf(u, nm1);
+                                // floor(u) sits in the low mantissa bits after a round-down add of 1.5 * 2^23
+                                const uint32_t bits = __float_as_uint(__fadd_rd(u, 12582912.0f));
+                                float kk, bb;
+                                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(kk), "=f"(bb) : "r"((bits << 7) + rep_lane));
+                                e[k] = __fmaf_rn(kk, x, bb);
+                            }
+                            sum0 += e[0] + e[4];
+                            sum1 += e[1] + e[5];
+                            sum2 += e[2] + e[6];
+                            sum3 += e[3] + e[7];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) pk[jj * 4 + k] = AT<T>::pack(e[2 * k], e[2 * k + 1]);
+                        }
                     }
-                    m = max3f(m, m0, m1);
-                }
-            } else {
-                asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
-            }
-        }
-        if constexpr (NG == 2) {   // the two groups saw different keys of the row
-            s_red[g2][row] = m;
-            asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-            m = fmaxf(s_red[0][row], s_red[1][row]);
-            asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-        }
-        const float neg_ms = -(m * a.scale);
-        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-        const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(g2 * PBUF + row * ROWB);
-        const uint32_t p_row = tmem_p + ((uint32_t)(q * 32) << 16);   // this warp's lane quarter of the P columns
-        // ---- sweep 2: e = PWL_exp(s - m), row sum, P tiles
-#pragma unroll 1
-        for (int j = 0; j < half; ++j) {
-            wait_all(&bar_s_full[g2], (uint32_t)((cnt1 + j) & 1));
-            if (ok) nm_tc_fence_after();
+                    // The stores wait until P V of the group's previous chunk has read the tile; that MMA was
+                    // issued just before this chunk began, so the first half's arithmetic runs ahead of it.
+                    if (hh == 0 && j >= 1) {
+                        wait_all(&bar_p_empty[g2], (pv_base + (uint32_t)(j - 1)) & 1u);
+                    }
+                    if (ok) {
+                        if constexpr (PT) {
+                            if (hh == 0 && j >= 1) nm_tc_fence_after();   // ordered after the P V that read the columns
+                            tmem_st16(p_row + (uint32_t)(hh * 16), pk);   // keys 32 hh .. 32 hh + 31 of this thread's row
+                        } else {
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                uint32_t r[32];
-                if (ok) {
-                    nm_tmem_ld32_sync(t_row + (uint32_t)(hh * 32), r);
+                            for (int jj = 0; jj < 4; ++jj) {
+                                // chunk index is XORed with the row (128-byte swizzle of the K-major P tile)
+                                const uint32_t addr = prow + (uint32_t)(((hh * 4 + jj) ^ (row & 7)) << 4);
+                                asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pk[jj * 4]), "r"(pk[jj * 4 + 1]),
+                                             "r"(pk[jj * 4 + 2]), "r"(pk[jj * 4 + 3])
+                                             : "memory");
+                            }
+                        }
+                    }
                 }
-                if (hh == 1) {
+                if constexpr (PT) {
+                    tmem_st_wait();          // the P columns are written
                     nm_tc_fence_before();
-                    asm volatile("bar.arrive %0, %1;" ::"r"(bar_sc), "n"(160) : "memory");
+                } else {
+                    nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
                 }
-                uint32_t pk[16];   // the half's 32 exponentials, packed to 16 bits
-                if (ok) {
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {   // 8 keys = one 16-byte chunk of the P row
-                        float e[8];
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const float x = __fmaf_rn(__uint_as_float(r[jj * 8 + k]), a.scale, neg_ms);
-                            float u = fmaxf(__fmaf_rn(x, inv_h, off), 0.0f);
-                            if (CLAMP_HI) u = fminf(u, nm1);
-                            // floor(u) sits in the low mantissa bits after a round-down add of 1.5 * 2^23
-                            const uint32_t bits = __float_as_uint(__fadd_rd(u, 12582912.0f));
-                            float kk, bb;
-                            asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(kk), "=f"(bb) : "r"((bits << 7) + rep_lane));
-                            e[k] = __fmaf_rn(kk, x, bb);
-                        }
-                        sum0 += e[0] + e[4];
-                        sum1 += e[1] + e[5];
-                        sum2 += e[2] + e[6];
-                        sum3 += e[3] + e[7];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) pk[jj * 4 + k] = AT<T>::pack(e[2 * k], e[2 * k + 1]);
-                    }
-                }
-                // The stores wait until P V of the group's previous chunk has read the tile; that MMA was
-                // issued just before this chunk began, so the first half's arithmetic runs ahead of it.
-                if (hh == 0 && j >= 1) {
-                    wait_all(&bar_p_empty[g2], (uint32_t)((j - 1) & 1));
-                }
-                if (ok) {
-                    if constexpr (PT) {
-                        if (hh == 0 && j >= 1) nm_tc_fence_after();   // ordered after the P V that read the columns
-                        tmem_st16(p_row + (uint32_t)(hh * 16), pk);   // keys 32 hh .. 32 hh + 31 of this thread's row
-                    } else {
-#pragma unroll
-                        for (int jj = 0; jj < 4; ++jj) {
-                            // chunk index is XORed with the row (128-byte swizzle of the K-major P tile)
-                            const uint32_t addr = prow + (uint32_t)(((hh * 4 + jj) ^ (row & 7)) << 4);
-                            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pk[jj * 4]), "r"(pk[jj * 4 + 1]),
-                                         "r"(pk[jj * 4 + 2]), "r"(pk[jj * 4 + 3])
-                                         : "memory");
-                        }
-                    }
-                }
+                asm volatile("bar.arrive %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");
             }
-            if constexpr (PT) {
-                tmem_st_wait();          // the P columns are written
-                nm_tc_fence_before();
-            } else {
-                nm_fence_proxy_async();   // generic-proxy writes of P become visible to the tensor core
+            float sum = (sum0 + sum1) + (sum2 + sum3);
+            if constexpr (NG == 2) {
+                s_red[g2][row] = sum;
+                asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+                sum = s_red[0][row] + s_red[1][row];
             }
-            asm volatile("bar.arrive %0, %1;" ::"r"(bar_pr), "n"(160) : "memory");
-        }
-        float sum = (sum0 + sum1) + (sum2 + sum3);
-        if constexpr (NG == 2) {
-            s_red[g2][row] = sum;
-            asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-            sum = s_red[0][row] + s_red[1][row];
-        }
-        // ---- r = PWL_recip(sigma), then (O_0 + O_1) * r; each group stores 32 of the 64 channels
-        const int sr = nm_pwl_index(sum, a.t_rcp->inv_h, a.t_rcp->off, (float)(a.t_rcp->n - 1));
-        const float2 kbr = a.t_rcp->kb[sr];
-        const float rinv = __fmaf_rn(kbr.x, sum, kbr.y);
+            // ---- r = PWL_recip(sigma), then (O_0 + O_1) * r; each group stores 32 of the 64 channels
+            const int sr = nm_pwl_index(sum, a.t_rcp->inv_h, a.t_rcp->off, (float)(a.t_rcp->n - 1));
+            const float2 kbr = a.t_rcp->kb[sr];
+            const float rinv = __fmaf_rn(kbr.x, sum, kbr.y);
 #pragma unroll
-        for (int gg = 0; gg < NG; ++gg)   // the last P V of every group has completed
-            wait_all(&bar_p_empty[gg], (uint32_t)((half - 1) & 1));
-        if (ok) {
-            nm_tc_fence_after();
+            for (int gg = 0; gg < NG; ++gg)   // the last P V of every group has completed
+                wait_all(&bar_p_empty[gg], (pv_base + (uint32_t)(half - 1)) & 1u);
+            pv_base += (uint32_t)half;
             constexpr int CH = HD / NG;   // channels this warp stores
+            if (ok) nm_tc_fence_after();
             T* orow = reinterpret_cast<T*>(a.out) + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
                       (size_t)g * HD + g2 * CH;
             const uint32_t o_addr = tmem_base + ((uint32_t)(q * 32) << 16) + O_OFF + (uint32_t)(g2 * CH);
 #pragma unroll
             for (int jj = 0; jj < CH / 16; ++jj) {   // 16 channels at a time, summed over the groups' accumulators
                 uint32_t r0[16], r1[16];
-                nm_tmem_ld16_sync(o_addr + (uint32_t)(jj * 16), r0);
-                if constexpr (NG == 2) nm_tmem_ld16_sync(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
-                float v[16];
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    float x = __uint_as_float(r0[k]);
-                    if constexpr (NG == 2) x += __uint_as_float(r1[k]);
-                    v[k] = x * rinv;
+                if (ok) {
+                    nm_tmem_ld16_sync(o_addr + (uint32_t)(jj * 16), r0);
+                    if constexpr (NG == 2) nm_tmem_ld16_sync(o_addr + GRP_COLS + (uint32_t)(jj * 16), r1);
                 }
-                if (a.out_q) {
-                    int8_t code[16];
+                if (jj == CH / 16 - 1 && more) {
+                    // all of O is in registers: the control warp may start the next tile's sweep 1 over [S_g | O_g]
+                    nm_tc_fence_before();
+                    asm volatile("bar.arrive %0, %1;" ::"r"(bar_oc), "n"(160) : "memory");
+                }
+                if (ok) {
+                    float v[16];
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) code[k] = nm_quant_i8(AT<T>::round(v[k]), a.q_inv_scale);
-                    int8_t* qrow = a.out_q + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
-                                   (size_t)g * HD + g2 * CH;
-                    reinterpret_cast<uint4*>(qrow)[jj] = *reinterpret_cast<const uint4*>(code);
-                } else {
-                    uint32_t w[8];
+                    for (int k = 0; k < 16; ++k) {
+                        float x = __uint_as_float(r0[k]);
+                        if constexpr (NG == 2) x += __uint_as_float(r1[k]);
+                        v[k] = x * rinv;
+                    }
+                    if (a.out_q) {
+                        int8_t code[16];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) w[k] = AT<T>::pack(v[2 * k], v[2 * k + 1]);
-                    reinterpret_cast<uint4*>(orow)[2 * jj] = make_uint4(w[0], w[1], w[2], w[3]);
-                    reinterpret_cast<uint4*>(orow)[2 * jj + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                        for (int k = 0; k < 16; ++k) code[k] = nm_quant_i8(AT<T>::round(v[k]), a.q_inv_scale);
+                        int8_t* qrow = a.out_q + ((size_t)b * L + (size_t)qb * BQ + row) * ((size_t)a.heads * HD) +
+                                       (size_t)g * HD + g2 * CH;
+                        reinterpret_cast<uint4*>(qrow)[jj] = *reinterpret_cast<const uint4*>(code);
+                    } else {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) w[k] = AT<T>::pack(v[2 * k], v[2 * k + 1]);
+                        reinterpret_cast<uint4*>(orow)[2 * jj] = make_uint4(w[0], w[1], w[2], w[3]);
+                        reinterpret_cast<uint4*>(orow)[2 * jj + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    }
                 }
             }
         }
@@ -553,8 +646,19 @@ nm_status launch(nm_ctx* ctx, const nm_attn_desc* d, cudaStream_t st, int8_t* ou
     auto kern = attention_stream_kernel<T, CLAMP_HI, NG>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return NM_ERR_CUDA;
-    const int64_t grid = (int64_t)d->B * d->heads * (d->L / BQ);
-    if (grid > 0x7fffffffLL) return NM_ERR_SHAPE;
+    const int64_t tiles = (int64_t)d->B * d->heads * (d->L / BQ);
+    if (tiles > 0x7fffffffLL) return NM_ERR_SHAPE;
+    int64_t grid = tiles;
+    if (NG == 1) {
+        // persistent: one resident wave of CTAs, each walking over tiles.  Three CTAs per SM by the launch bounds
+        // (registers) and by tensor memory (3 x 160 of 512 columns); fewer if the exp table makes the shared
+        // memory larger (233472 bytes per SM, 1 KB reserved per CTA).
+        int64_t per_sm = 233472 / (int64_t)(smem + 1024 + 1536);
+        if (per_sm > 3) per_sm = 3;
+        if (per_sm < 1) per_sm = 1;
+        const int64_t cap = (int64_t)ctx->sm_count * per_sm;
+        if (grid > cap) grid = cap;
+    }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid);
@@ -588,15 +692,10 @@ nm_status nm_launch_attention_stream(nm_ctx* ctx, const nm_attn_desc* d, cudaStr
     if (!nm_attention_stream_supported(d)) return NM_ERR_UNSUPPORTED;
     // the softmax input is never positive: a table whose range reaches 0 needs no upper clamp
     const bool clamp_hi = ctx->h_tables[d->exp_slot].x_max < 0.0f;
-    // one group per CTA (three CTAs per SM, P through tensor memory) measures faster at every length tried
-    // (L = 128 ... 2048: 10 % at 512 and 2048); the two-group form stays selectable for comparison
-    const int groups = ctx->attn_groups ? ctx->attn_groups : 1;
-    if (groups == 1) {
-        if (d->dtype == NM_BF16)
-            return clamp_hi ? launch<__nv_bfloat16, true, 1>(ctx, d, st, out_q, q_inv_scale) : launch<__nv_bfloat16, false, 1>(ctx, d, st, out_q, q_inv_scale);
-        return clamp_hi ? launch<__half, true, 1>(ctx, d, st, out_q, q_inv_scale) : launch<__half, false, 1>(ctx, d, st, out_q, q_inv_scale);
-    }
+    // One softmax group per CTA: three persistent CTAs per SM with P through tensor memory.  (The kernel text
+    // still carries the two-group form, NG = 2, which splits the keys of a tile between two pipelines of one
+    // CTA; it measured slower at every length from 128 to 2048 once P left shared memory, and is not built.)
     if (d->dtype == NM_BF16)
-        return clamp_hi ? launch<__nv_bfloat16, true, 2>(ctx, d, st, out_q, q_inv_scale) : launch<__nv_bfloat16, false, 2>(ctx, d, st, out_q, q_inv_scale);
-    return clamp_hi ? launch<__half, true, 2>(ctx, d, st, out_q, q_inv_scale) : launch<__half, false, 2>(ctx, d, st, out_q, q_inv_scale);
+        return clamp_hi ? launch<__nv_bfloat16, true, 1>(ctx, d, st, out_q, q_inv_scale) : launch<__nv_bfloat16, false, 1>(ctx, d, st, out_q, q_inv_scale);
+    return clamp_hi ? launch<__half, true, 1>(ctx, d, st, out_q, q_inv_scale) : launch<__half, false, 1>(ctx, d, st, out_q, q_inv_scale);
 }

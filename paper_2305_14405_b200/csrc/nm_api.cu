@@ -118,8 +118,6 @@ nm_status nm_ctx_create(nm_ctx** out, int device)
         ctx->pdl = (e && e[0] == '0') ? 0 : 1;
         e = getenv("NM_ATTN_RESIDENT");     // NM_ATTN_RESIDENT=1: algo 0 picks the resident-score attention kernel
         ctx->attn_resident = (e && e[0] == '1') ? 1 : 0;
-        e = getenv("NM_ATTN_GROUPS");       // NM_ATTN_GROUPS=1|2: softmax groups per CTA of the streaming kernel
-        ctx->attn_groups = (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;   // 0: chosen by sequence length
     }
     ctx->prof = new (std::nothrow) NmProfRecord[NM_PROF_MAX];
     if (!ctx->prof) { cudaFree(ctx->d_tables); cudaFree(ctx->d_status); cudaFree(ctx->d_pool_w); delete ctx; return NM_ERR_CUDA; }

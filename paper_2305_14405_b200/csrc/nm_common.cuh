@@ -45,7 +45,6 @@ struct nm_ctx {
     NmProfRecord* prof;        // NM_PROF_MAX records, host memory
     int pdl;                   // launch kernels with programmatic stream serialization (prologue overlap)
     int attn_resident;         // algo 0 prefers the attention kernel with the score block resident in TMEM
-    int attn_groups;           // softmax groups per CTA of the streaming attention kernel (1 or 2; 0 = pick)
     void* static_ws;           // device address of the library's fixed scratch array on this device (or null)
     void* d_pool_w;            // 64 x 64 matrix (1/HW on the diagonal) of the average pool run as a GEMM; 8 KB
     int pool_w_hw, pool_w_dtype;   // what d_pool_w currently holds (0 = nothing)

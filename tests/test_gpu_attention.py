@@ -58,19 +58,22 @@ def test_attention_bf16(nm, ctx, algo, B, L, h, d, qk):
     assert_close_bf16(got, ref, "attention bf16 %s" % algo)
 
 
-@pytest.mark.parametrize("groups", ["1", "2"])
 @pytest.mark.parametrize("dtype", ["bf16", "f16"])
 @pytest.mark.parametrize("B,L,h", [(2, 128, 3), (1, 384, 2), (1, 640, 1)])
-def test_attention_stream_groups(nm, monkeypatch, groups, dtype, B, L, h):
-    """The streaming kernel with one and with two softmax groups per CTA (the library picks by
-    sequence length; NM_ATTN_GROUPS, read when a context is created, forces either)."""
-    monkeypatch.setenv("NM_ATTN_GROUPS", groups)
-    c = nm.Context(0)
-    try:
-        got, ref = run(nm, c, dtype, B, L, h, 64, nm.ALGO_TC, seed=17 + L, qk_scale=0.8)
-    finally:
-        c.close()
-    assert_close_bf16(got, ref, "attention %s, %s group(s), L=%d" % (dtype, groups, L))
+def test_attention_stream_lengths(nm, ctx, dtype, B, L, h):
+    """The streaming kernel at lengths with an odd and an even number of 128-key chunks."""
+    got, ref = run(nm, ctx, dtype, B, L, h, 64, nm.ALGO_TC, seed=17 + L, qk_scale=0.8)
+    assert_close_bf16(got, ref, "attention %s, L=%d" % (dtype, L))
+
+
+@pytest.mark.parametrize("B,L,h", [(10, 128, 50), (4, 384, 40), (3, 640, 31)])
+def test_attention_stream_several_tiles_per_cta(nm, ctx, B, L, h):
+    """More (batch, head, query block) tiles than resident CTAs (3 per SM), so that every CTA walks over
+    several tiles; the lengths give an odd number of barrier phases per tile (3, 9 and 15 score products),
+    which the running phase counters must carry from tile to tile."""
+    assert B * h * (L // 128) > 3 * torch.cuda.get_device_properties(0).multi_processor_count
+    got, ref = run(nm, ctx, "bf16", B, L, h, 64, nm.ALGO_TC, seed=5 + L, qk_scale=0.8)
+    assert_close_bf16(got, ref, "attention, %d tiles, L=%d" % (B * h * (L // 128), L))
 
 
 @pytest.mark.parametrize("n", [16, 256])
