@@ -9,8 +9,14 @@
 // this kernel computes Q K^T TWICE: a first sweep over the keys only for the row maximum, a second
 // sweep for the exponentials.  The tensor pipe is idle most of the time in this ALU-bound kernel, so
 // the second Q K^T is free, and the footprint drops to 128 tensor-memory columns and ~50 KB of
-// shared memory per softmax group (plus Q and the table): two or three CTAs fit on an SM and one
+// shared memory per softmax group (plus Q and the table): three CTAs fit on an SM and one
 // CTA's loads, MMAs and hand-offs overlap the others' arithmetic.  Any L that is a multiple of 128.
+//
+// CTAs are persistent: one resident wave (three per SM) walks over the (batch, head, 128-query block) tiles.
+// Barriers, tensor memory and the replicated table are set up once per CTA; every mbarrier's phase is a running
+// count carried from tile to tile; after a tile's last Q K^T the control warp already fetches the next tile's Q
+// and first K chunks, after its last P V the next first V chunk, and the next tile's first product starts as
+// soon as the softmax warps have read the accumulator out of tensor memory.
 //
 // The 16-bit P tile of the one-group form never touches shared memory: the softmax warps write it to 32 further
 // tensor-memory columns (tcgen05.st) and P V takes its A operand from there; the shared-memory pipe, which the
@@ -18,7 +24,8 @@
 //
 // A group is one control warp and four softmax warps, an independent pipeline that owns 128
 // tensor-memory columns [S_g | O_g], two K stages, a V stage and a P tile.  A CTA has NG = 1 or 2
-// groups (template parameter); with two, the groups split the keys: in sweep 1 group g takes the
+// groups (template parameter; only NG = 1 is built, see nm_launch_attention_stream); with two, the groups split
+// the keys: in sweep 1 group g takes the
 // 128-key chunks g, g+NG, ... (scores over all 128 columns, K staged in its two K stages and,
 // alternately, in its P tile); in sweep 2 the 64-key chunks g, g+NG, ... (scores in S_g, accumulator
 // O_g); row maxima and sums are exchanged through shared memory and the accumulators summed in the
