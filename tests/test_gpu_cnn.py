@@ -164,6 +164,38 @@ def test_resnet50_two_images(nm, ctx, random_bn):
     assert np.all(np.isfinite(got)) and not (err > bound).any(), "%d outside" % (err > bound).sum()
 
 
+def test_resnet50_host_entry_points_two_streams(nm, ctx):
+    """The host-buffer forms: the blocking call equals the device-resident forward bit for bit, and four
+    asynchronous calls alternating between two streams (own device buffers and workspaces, different images
+    per call) equal the blocking call's results."""
+    from paper_2305_14405_b200.harness_cnn import Resnet50Model
+    relu_tables(ctx)
+    x, convs, fc_w, fc_b = nm_inputs_cnn.resnet50_inputs(2, seed=3, random_bn=True)
+    m = Resnet50Model(ctx, 2, convs, fc_w, fc_b)
+    base = torch.from_numpy(x).half()
+    xs = [(base * (1.0 - 0.1 * i)).pin_memory() for i in range(4)]
+    xd = torch.empty(base.shape, dtype=torch.float16, device="cuda")
+    ld = torch.empty((2, fc_w.shape[0]), dtype=torch.float16, device="cuda")
+    want = []
+    for xh in xs:
+        lh = torch.empty((2, fc_w.shape[0]), dtype=torch.float16).pin_memory()
+        ctx.resnet50_forward_host(m.array, m.fc_w, m.fc_b, m.cfg, xh, lh, xd, ld, m.workspace)
+        want.append(lh.clone())
+    assert torch.equal(want[0], m.forward(xs[0].cuda()).cpu())
+    slots = [(torch.empty_like(xd), torch.empty_like(ld), torch.empty_like(m.workspace), torch.cuda.Stream())
+             for _ in range(2)]
+    outs = [torch.empty_like(want[0]).pin_memory() for _ in range(4)]
+    torch.cuda.synchronize()
+    for i, xh in enumerate(xs):
+        sx, sl, ws, st = slots[i % 2]
+        ctx.resnet50_forward_host(m.array, m.fc_w, m.fc_b, m.cfg, xh, outs[i], sx, sl, ws, stream=st, wait=False)
+    torch.cuda.synchronize()
+    ctx.check_device_status()
+    for i in range(4):
+        assert torch.equal(outs[i], want[i]), i
+    assert not torch.equal(want[0], want[1])
+
+
 def test_resnet50_full_batch_sampled_images(nm, ctx):
     """Config 5 in the benchmark's launch configuration (batch 128, fp16 NHWC, random folded BatchNorm):
     images are independent, so the oracle runs two sampled images through the whole network."""
