@@ -68,6 +68,21 @@ def test_int8_attention_full_size_sampled(nm, ctx):
         assert np.array_equal(got[b * L:(b + 1) * L].view(np.uint32), ref.view(np.uint32)), "batch %d" % b
 
 
+@pytest.mark.parametrize("B,L,h", [(10, 128, 50), (4, 384, 40)])
+def test_int8_attention_several_tiles_per_cta(nm, ctx, B, L, h):
+    """More tiles than resident CTAs (3 per SM), lengths with an odd number of barrier phases per tile (3 and 9
+    score products): the persistent CTAs carry their phase counts from tile to tile.  fp32 output bit for bit."""
+    d = 64
+    assert B * h * (L // 128) > 3 * torch.cuda.get_device_properties(0).multi_processor_count
+    tabs = load_tables_both(ctx, 64, {"exp": (-8.0, 0.0), "recip": (L / 16.0, float(L))})
+    codes, s_qk, s_v = _codes(B, L, h, d, 41 + L, 0.7)
+    out = torch.full((B * L, h * d), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.attention_pwl_i8(torch.from_numpy(codes).cuda(), out, B, L, h, d, s_qk, s_qk, s_v)
+    ctx.check_device_status()
+    ref = oracle.attention_i8(codes, B, L, h, d, s_qk, s_qk, s_v, tabs["exp"], tabs["recip"])
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
 def test_int8_attention_argument_errors(nm, ctx):
     load_tables_both(ctx, 64, {"exp": (-8.0, 0.0), "recip": (8.0, 128.0)})
     q = torch.zeros(128, 192, dtype=torch.int8, device="cuda")
