@@ -46,6 +46,8 @@ def parse_args():
                    help="rows workload: LayerNorm as PWL_recip(PWL_sqrt(v + eps)) instead of one rsqrt table")
     p.add_argument("--hidden", type=int, default=0, help="encoder workloads: override H (heads = H/64, F = 4H)")
     p.add_argument("--layers", type=int, default=0, help="encoder workloads: override the number of layers")
+    p.add_argument("--resnet-blocks", default="", help="c5: bottleneck blocks per stage, e.g. 3,4,23,3 (default 3,4,6,3)")
+    p.add_argument("--resnet-width", type=int, default=0, help="c5: width of the first stage (default 64)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-rows-leg", action="store_true",
                    help="encoder workloads: skip the row-kernel bandwidth leg on a tensor beyond L2")
@@ -309,21 +311,27 @@ class ResnetWorkload:
         self.args = args
         self.batch = args.batch or 128
         self.units_per_step = self.batch
+        self.blocks = tuple(int(v) for v in args.resnet_blocks.split(",")) if args.resnet_blocks else (3, 4, 6, 3)
+        assert len(self.blocks) == 4, "--resnet-blocks takes four numbers"
+        self.base = args.resnet_width or 64
+        self.variant = self.blocks != (3, 4, 6, 3) or self.base != 64
 
     def config(self, world):
-        return {"workload": "c5_resnet50_f16", "batch": self.batch, "image": "224x224x3 NHWC", "convolutions": 53,
+        name = "c5_resnet50_f16" if not self.variant else "c5_resnet_b%s_w%d_f16" % ("-".join(map(str, self.blocks)), self.base)
+        return {"workload": name, "batch": self.batch, "image": "224x224x3 NHWC",
+                "blocks": list(self.blocks), "base_width": self.base, "convolutions": 1 + sum(3 * b + 1 for b in self.blocks),
                 "classes": 1000, "batchnorm": "folded into weights and biases", "relu": "2-segment PWL table",
                 "seed": self.args.seed, "parallelism": "replicas" if world > 1 else "single",
                 "l2": "activations (up to %.0f MB per layer at this batch) exceed the 126 MB L2; no flush"
-                      % (self.batch * 112 * 112 * 64 * 2 / 1e6)}
+                      % (self.batch * 112 * 112 * self.base * 2 / 1e6)}
 
     def flops_per_step(self):
         import nm_inputs_cnn
-        specs = iter(nm_inputs_cnn.resnet50_conv_specs())
+        specs = iter(nm_inputs_cnn.resnet_conv_specs(self.blocks, self.base))
         cin, cout, k, _, _ = next(specs)
         total = 2 * 112 * 112 * cout * k * k * cin
         h = 56
-        for st, nb in enumerate(nm_inputs_cnn.STAGE_BLOCKS):
+        for st, nb in enumerate(self.blocks):
             for b in range(nb):
                 stride = 2 if (b == 0 and st > 0) else 1
                 ho = h // stride
@@ -333,7 +341,7 @@ class ResnetWorkload:
                     cd = next(specs)
                     total += 2 * ho * ho * cd[1] * cd[0]
                 h = ho
-        total += 2 * 2048 * 1000
+        total += 2 * 32 * self.base * 1000
         return total * self.batch
 
     def setup(self, ctx, dev, rank):
@@ -344,13 +352,14 @@ class ResnetWorkload:
         ctx.load_function_table(nm.SLOT_RELU, nm.FUNC_RELU, 2, -8.0, 8.0)
         # the same model on every replica (seed), its own images per rank (seed + rank)
         self.x_np, self.convs, self.fc_w, self.fc_b = nm_inputs_cnn.resnet50_inputs(
-            self.batch, seed=self.args.seed, random_bn=True)
+            self.batch, seed=self.args.seed, random_bn=True, blocks=self.blocks, base_width=self.base)
         if rank > 0:
             import numpy as np
             import nm_inputs
             rng = np.random.default_rng(self.args.seed + rank)
             self.x_np = nm_inputs.round_to(rng.random(self.x_np.shape, dtype=np.float32), "f16")
-        self.model = Resnet50Model(ctx, self.batch, self.convs, self.fc_w, self.fc_b, device=dev, algo=self.args.algo)
+        self.model = Resnet50Model(ctx, self.batch, self.convs, self.fc_w, self.fc_b, device=dev, algo=self.args.algo,
+                                   blocks=self.blocks, base_width=self.base)
         self.x = torch.from_numpy(self.x_np).to(dev).half()
         self.y = torch.empty((self.batch, 1000), dtype=torch.float16, device=dev)
         self.xh = torch.from_numpy(self.x_np).half().pin_memory()
@@ -391,7 +400,7 @@ class ResnetWorkload:
         import oracle.cnn
         relu = oracle.Table.secant(oracle.RELU, 2, -8.0, 8.0)
         t0 = time.perf_counter()
-        oracle.cnn.resnet50(self.x_np[:n_img], self.convs, self.fc_w, self.fc_b, relu)
+        oracle.cnn.resnet50(self.x_np[:n_img], self.convs, self.fc_w, self.fc_b, relu, blocks=self.blocks)
         return time.perf_counter() - t0, oracle.num_threads()
 
     def cpu_baseline(self):

@@ -382,7 +382,17 @@ typedef struct {
     int32_t relu_slot;
     int32_t num_classes;
     int32_t algo;
+    /* Variants of the network (Section 5 compares ResNet-50 "and its variant models" by depth and width): the
+     * number of bottleneck blocks of the four stages and the width of the first stage (stage s has inner width
+     * base_width << s and 4x that many output channels; the stem has base_width channels).  All zero = ResNet-50:
+     * blocks {3, 4, 6, 3}, base_width 64.  blocks in 1..64; base_width a multiple of 8 in 8..256 (multiples of 64
+     * take the implicit-GEMM convolutions throughout).  convs then holds 1 + sum over stages of (3 blocks + 1)
+     * entries (nm_resnet_conv_count) and fc_w is [num_classes, 32 * base_width]. */
+    int32_t blocks[4];
+    int32_t base_width;
 } nm_resnet50_cfg;
+/* Entries of `convs` for a configuration (53 for ResNet-50); 0 if the configuration is not valid. */
+int32_t nm_resnet_conv_count(const nm_resnet50_cfg* cfg);
 size_t nm_resnet50_workspace_bytes(const nm_resnet50_cfg* cfg);
 nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w, const float* fc_b,
                               const nm_resnet50_cfg* cfg, const void* x, void* logits, void* workspace,

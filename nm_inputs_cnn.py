@@ -19,13 +19,15 @@ STAGE_BLOCKS = (3, 4, 6, 3)
 STAGE_WIDTH = (64, 128, 256, 512)
 
 
-def resnet50_conv_specs():
-    """(Cin, Cout, k, stride, pad) of the 53 convolutions in network order: conv1, then per block
-    conv_a (1x1), conv_b (3x3, carries the stride), conv_c (1x1) and, in the first block of a stage,
-    the 1x1 projection shortcut."""
-    specs = [(3, 64, 7, 2, 3)]
-    cin = 64
-    for st, (nb, width) in enumerate(zip(STAGE_BLOCKS, STAGE_WIDTH)):
+def resnet_conv_specs(blocks=STAGE_BLOCKS, base_width=64):
+    """(Cin, Cout, k, stride, pad) of the convolutions of a bottleneck ResNet in network order: conv1, then
+    per block conv_a (1x1), conv_b (3x3, carries the stride), conv_c (1x1) and, in the first block of a stage,
+    the 1x1 projection shortcut.  blocks: bottleneck blocks per stage; base_width: inner width of stage 1
+    (stage s: base_width << s).  (3, 4, 6, 3) and 64 give ResNet-50's 53 convolutions."""
+    specs = [(3, base_width, 7, 2, 3)]
+    cin = base_width
+    for st, nb in enumerate(blocks):
+        width = base_width << st
         for b in range(nb):
             stride = 2 if (b == 0 and st > 0) else 1
             specs.append((cin, width, 1, 1, 0))
@@ -34,17 +36,25 @@ def resnet50_conv_specs():
             if b == 0:
                 specs.append((cin, 4 * width, 1, stride, 0))
             cin = 4 * width
+    return specs
+
+
+def resnet50_conv_specs():
+    specs = resnet_conv_specs()
     assert len(specs) == 53
     return specs
 
 
-def resnet50_inputs(batch, seed=0, random_bn=False, num_classes=1000, image=224, dtype="f16"):
+def resnet50_inputs(batch, seed=0, random_bn=False, num_classes=1000, image=224, dtype="f16", blocks=STAGE_BLOCKS,
+                    base_width=64):
     """Returns (x [batch,image,image,3] fp32 holding dtype-rounded values in [0,1),
-    convs: list of dicts {w [Cout,k,k,Cin], b [Cout], spec}, fc_w [classes,2048], fc_b [classes])."""
+    convs: list of dicts {w [Cout,k,k,Cin], b [Cout], spec}, fc_w [classes, 32 base_width], fc_b [classes]).
+    blocks / base_width: the depth and width variants of the network (defaults: ResNet-50)."""
     rng = np.random.default_rng(seed)
     x = round_to(rng.random((batch, image, image, 3), dtype=np.float32), dtype)
     convs = []
-    for (cin, cout, k, stride, pad) in resnet50_conv_specs():
+    feat = 32 * base_width
+    for (cin, cout, k, stride, pad) in resnet_conv_specs(blocks, base_width):
         fan_in = cin * k * k
         w = (np.sqrt(2.0 / fan_in) * rng.standard_normal((cout, k, k, cin), dtype=np.float32)).astype(np.float32)
         if random_bn:
@@ -58,6 +68,6 @@ def resnet50_inputs(batch, seed=0, random_bn=False, num_classes=1000, image=224,
         else:
             b = np.zeros(cout, np.float32)
         convs.append({"w": round_to(w, dtype), "b": b, "spec": (cin, cout, k, stride, pad)})
-    fc_w = round_to((np.sqrt(1.0 / 2048) * rng.standard_normal((num_classes, 2048), dtype=np.float32)), dtype)
+    fc_w = round_to((np.sqrt(1.0 / feat) * rng.standard_normal((num_classes, feat), dtype=np.float32)), dtype)
     fc_b = (0.01 * rng.standard_normal(num_classes)).astype(np.float32)
     return x, convs, fc_w, fc_b

@@ -11,10 +11,12 @@ from . import Table, conv2d_nhwc, maxpool_nhwc, avgpool_nhwc, linear, pwl_eval
 STAGE_BLOCKS = (3, 4, 6, 3)
 
 
-def resnet50(x, convs, fc_w, fc_b, relu: Table, collect=None):
-    """x [N,H,W,3]; convs: 53 dicts with 'w', 'b', 'spec' = (Cin, Cout, k, stride, pad) in network
-    order (conv1; per block conv_a, conv_b, conv_c, and the projection in a stage's first block).
-    Returns logits [N, classes].  `collect`, if a list, receives the output of every block."""
+def resnet50(x, convs, fc_w, fc_b, relu: Table, collect=None, blocks=STAGE_BLOCKS):
+    """x [N,H,W,3]; convs: dicts with 'w', 'b', 'spec' = (Cin, Cout, k, stride, pad) in network
+    order (conv1; per block conv_a, conv_b, conv_c, and the projection in a stage's first block): 53 for
+    ResNet-50.  `blocks`: bottleneck blocks per stage, for the depth variants Section 5 compares (the widths
+    are those of the weights).  Returns logits [N, classes].  `collect`, if a list, receives the output of
+    every block."""
     it = iter(convs)
 
     def conv(inp, c, table, residual=None):
@@ -23,7 +25,7 @@ def resnet50(x, convs, fc_w, fc_b, relu: Table, collect=None):
 
     y = conv(x, next(it), relu)
     y = maxpool_nhwc(y, 3, 2, 1)
-    for st, nb in enumerate(STAGE_BLOCKS):
+    for st, nb in enumerate(blocks):
         for b in range(nb):
             ca, cb, cc = next(it), next(it), next(it)
             t = conv(y, ca, relu)
@@ -33,5 +35,6 @@ def resnet50(x, convs, fc_w, fc_b, relu: Table, collect=None):
             y = pwl_eval(relu, z)[0]                        # ReLU after the add
             if collect is not None:
                 collect.append(y)
+    assert next(it, None) is None, "more convolutions than the block counts use"
     pooled = avgpool_nhwc(y)
     return linear(pooled, fc_w, fc_b)

@@ -31,6 +31,7 @@ EXPORTS = [
     "nm_conv2d_workspace_bytes", "nm_conv2d_pwl", "nm_maxpool2d", "nm_maxpool2d_pwl", "nm_avgpool_global", "nm_resnet50_workspace_bytes",
     "nm_resnet50_forward", "nm_resnet50_forward_host", "nm_pwl_table_build_elastic",
     "nm_selftest_bounded_wait", "nm_attention_pwl_i8", "nm_encoder_stack_host_async", "nm_resnet50_forward_host_async",
+    "nm_resnet_conv_count",
 ]
 KERNEL_KINDS = ("pwl_apply", "layernorm", "quantize", "linear_simt", "linear_tc", "attention_simt", "attention_tc",
                 "im2col", "pool")
@@ -88,7 +89,7 @@ class ConvParams(C.Structure):
 
 class Resnet50Cfg(C.Structure):
     _fields_ = [("batch", C.c_int32), ("dtype", C.c_int), ("relu_slot", C.c_int32), ("num_classes", C.c_int32),
-                ("algo", C.c_int32)]
+                ("algo", C.c_int32), ("blocks", C.c_int32 * 4), ("base_width", C.c_int32)]
 
 
 class EncoderCfg(C.Structure):
@@ -160,6 +161,8 @@ def load():
                                              C.POINTER(Resnet50Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_size_t, C.c_void_p]
     lib.nm_resnet50_forward_host_async.argtypes = lib.nm_resnet50_forward_host.argtypes
+    lib.nm_resnet_conv_count.restype = C.c_int32
+    lib.nm_resnet_conv_count.argtypes = [C.POINTER(Resnet50Cfg)]
     lib.nm_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.nm_ctx_profile_enable.argtypes = [C.c_void_p, C.c_int]
     lib.nm_ctx_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_double),
@@ -404,10 +407,19 @@ class Context:
                "nm_avgpool_global")
 
     @staticmethod
-    def resnet50_cfg(batch, dtype, num_classes=1000, relu_slot=SLOT_RELU, algo=ALGO_AUTO):
+    def resnet50_cfg(batch, dtype, num_classes=1000, relu_slot=SLOT_RELU, algo=ALGO_AUTO, blocks=None, base_width=0):
+        """blocks: bottleneck blocks of the four stages (None: ResNet-50's 3, 4, 6, 3); base_width: width of the
+        first stage (0: 64)."""
         c = Resnet50Cfg()
         c.batch, c.dtype, c.relu_slot, c.num_classes, c.algo = batch, dtype, relu_slot, num_classes, algo
+        if blocks is not None:
+            for i in range(4):
+                c.blocks[i] = blocks[i]
+        c.base_width = base_width
         return c
+
+    def resnet_conv_count(self, cfg) -> int:
+        return int(self._lib.nm_resnet_conv_count(C.byref(cfg)))
 
     def resnet50_workspace_bytes(self, cfg) -> int:
         return int(self._lib.nm_resnet50_workspace_bytes(C.byref(cfg)))

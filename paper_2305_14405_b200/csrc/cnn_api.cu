@@ -62,8 +62,22 @@ bool conv_geom(const nm_conv_desc* d, ConvGeom* g)
 }
 
 // stage widths and block counts of the ResNet-50 topology
-const int kStageBlocks[4] = {3, 4, 6, 3};
-const int kStageWidth[4] = {64, 128, 256, 512};
+// depth per stage and first-stage width of a configuration (zeros: ResNet-50); false if not valid
+struct ResnetShape {
+    int blocks[4];
+    int base;
+};
+bool resnet_shape(const nm_resnet50_cfg* c, ResnetShape* sh)
+{
+    const int def_blocks[4] = {3, 4, 6, 3};
+    const bool all_zero = c->blocks[0] == 0 && c->blocks[1] == 0 && c->blocks[2] == 0 && c->blocks[3] == 0;
+    for (int i = 0; i < 4; ++i) {
+        sh->blocks[i] = all_zero ? def_blocks[i] : c->blocks[i];
+        if (sh->blocks[i] < 1 || sh->blocks[i] > 64) return false;
+    }
+    sh->base = c->base_width == 0 ? 64 : c->base_width;
+    return sh->base >= 8 && sh->base <= 256 && sh->base % 8 == 0;
+}
 
 }  // namespace
 
@@ -219,14 +233,16 @@ nm_status nm_avgpool_global(nm_ctx* ctx, const void* x, void* y, nm_dtype dtype,
     return nm_launch_conv_tc(ctx, &c, st);
 }
 
-// Workspace: four activation buffers of the largest activation (batch x 112 x 112 x 64 =
-// batch x 56 x 56 x 256 elements), one pooled vector, and the largest gather buffer (conv1).
-static void resnet_layout(const nm_resnet50_cfg* c, size_t* act, size_t* pooled, size_t* gather, size_t* total)
+// Workspace: four activation buffers of the largest activation (batch x 112 x 112 x base =
+// batch x 56 x 56 x 4 base elements), one pooled vector, and the largest gather buffer (conv1).
+static void resnet_layout(const nm_resnet50_cfg* c, const ResnetShape& sh, size_t* act, size_t* pooled, size_t* gather,
+                          size_t* total)
 {
-    *act = align256((size_t)c->batch * 112 * 112 * 64 * 2);
-    *pooled = align256((size_t)c->batch * 2048 * 2);
-    size_t g = align256((size_t)c->batch * 112 * 112 * 152 * 2) + align256((size_t)64 * 152 * 2);  // conv1: K 147 -> 152
-    const size_t g3 = align256((size_t)c->batch * 56 * 56 * 576 * 2);                              // stage-1 3x3
+    const size_t base = (size_t)sh.base;
+    *act = align256((size_t)c->batch * 112 * 112 * base * 2);
+    *pooled = align256((size_t)c->batch * 32 * base * 2);
+    size_t g = align256((size_t)c->batch * 112 * 112 * 152 * 2) + align256(base * 152 * 2);  // conv1: K 147 -> 152
+    const size_t g3 = align256((size_t)c->batch * 56 * 56 * 9 * base * 2);                   // stage-1 3x3
     if (g3 > g) g = g3;
     *gather = g;
     *total = 4 * *act + *pooled + *gather;
@@ -234,10 +250,20 @@ static void resnet_layout(const nm_resnet50_cfg* c, size_t* act, size_t* pooled,
 
 size_t nm_resnet50_workspace_bytes(const nm_resnet50_cfg* cfg)
 {
-    if (!cfg || cfg->batch < 1) return 0;
+    ResnetShape sh;
+    if (!cfg || cfg->batch < 1 || !resnet_shape(cfg, &sh)) return 0;
     size_t act, pooled, gather, total;
-    resnet_layout(cfg, &act, &pooled, &gather, &total);
+    resnet_layout(cfg, sh, &act, &pooled, &gather, &total);
     return total;
+}
+
+int32_t nm_resnet_conv_count(const nm_resnet50_cfg* cfg)
+{
+    ResnetShape sh;
+    if (!cfg || !resnet_shape(cfg, &sh)) return 0;
+    int n = 1;
+    for (int st = 0; st < 4; ++st) n += 3 * sh.blocks[st] + 1;
+    return n;
 }
 
 nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const void* fc_w, const float* fc_b,
@@ -247,8 +273,11 @@ nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const vo
     if (!ctx || !convs || !fc_w || !cfg || !x || !logits) return NM_ERR_INVALID_ARG;
     if (cfg->batch < 1 || cfg->num_classes < 8 || cfg->num_classes % 8 != 0) return NM_ERR_SHAPE;
     if (cfg->dtype != NM_F16 && cfg->dtype != NM_BF16) return NM_ERR_UNSUPPORTED;
+    ResnetShape sh;
+    if (!resnet_shape(cfg, &sh)) return NM_ERR_SHAPE;
+    const int base = sh.base, n_convs = nm_resnet_conv_count(cfg);
     size_t act, pooled, gather, total;
-    resnet_layout(cfg, &act, &pooled, &gather, &total);
+    resnet_layout(cfg, sh, &act, &pooled, &gather, &total);
     if (!workspace || ws_bytes < total) return NM_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return NM_ERR_ALIGNMENT;
     uint8_t* ws = (uint8_t*)workspace;
@@ -271,15 +300,15 @@ nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const vo
     };
 
     // stem: 7x7/2 convolution + ReLU, 3x3/2 max-pool
-    nm_status s = conv(x, 224, 224, 3, 64, 7, 2, 3, nullptr, 0, buf[0]);
+    nm_status s = conv(x, 224, 224, 3, base, 7, 2, 3, nullptr, 0, buf[0]);
     if (s != NM_OK) return s;
-    s = nm_maxpool2d(ctx, buf[0], buf[1], cfg->dtype, Nb, 112, 112, 64, 3, 2, 1, stream);
+    s = nm_maxpool2d(ctx, buf[0], buf[1], cfg->dtype, Nb, 112, 112, base, 3, 2, 1, stream);
     if (s != NM_OK) return s;
     int cur = 1;  // buffer holding the block input
-    int H = 56, Cin = 64;
+    int H = 56, Cin = base;
     for (int st = 0; st < 4; ++st) {
-        const int width = kStageWidth[st], Cout = 4 * width;
-        for (int b = 0; b < kStageBlocks[st]; ++b) {
+        const int width = base << st, Cout = 4 * width;
+        for (int b = 0; b < sh.blocks[st]; ++b) {
             const int stride = (b == 0 && st > 0) ? 2 : 1;
             const int Ho = H / stride;
             // the three free buffers
@@ -323,14 +352,15 @@ nm_status nm_resnet50_forward(nm_ctx* ctx, const nm_conv_params* convs, const vo
             Cin = Cout;
         }
     }
-    if (ci != NM_RESNET50_CONVS) return NM_ERR_INVALID_ARG;
-    s = nm_avgpool_global(ctx, buf[cur], pool_buf, cfg->dtype, Nb, 7, 7, 2048, stream);
+    if (ci != n_convs) return NM_ERR_INVALID_ARG;
+    const int feat = 32 * base;   // channels of the last stage
+    s = nm_avgpool_global(ctx, buf[cur], pool_buf, cfg->dtype, Nb, 7, 7, feat, stream);
     if (s != NM_OK) return s;
     nm_linear_desc ld;
     memset(&ld, 0, sizeof(ld));
-    ld.M = Nb; ld.N = cfg->num_classes; ld.K = 2048;
+    ld.M = Nb; ld.N = cfg->num_classes; ld.K = feat;
     ld.in_dtype = cfg->dtype; ld.out_dtype = cfg->dtype;
-    ld.A = pool_buf; ld.lda = 2048; ld.W = fc_w; ld.ldw = 2048; ld.bias = fc_b;
+    ld.A = pool_buf; ld.lda = feat; ld.W = fc_w; ld.ldw = feat; ld.bias = fc_b;
     ld.slot = NM_SLOT_NONE; ld.out = logits; ld.ldo = cfg->num_classes; ld.algo = cfg->algo;
     return nm_linear_pwl(ctx, &ld, stream);
 }

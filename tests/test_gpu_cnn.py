@@ -164,6 +164,35 @@ def test_resnet50_two_images(nm, ctx, random_bn):
     assert np.all(np.isfinite(got)) and not (err > bound).any(), "%d outside" % (err > bound).sum()
 
 
+@pytest.mark.parametrize("blocks,base", [((1, 1, 1, 1), 64), ((2, 1, 2, 1), 128), ((1, 2, 1, 1), 32)])
+def test_resnet_variants(nm, ctx, blocks, base):
+    """Depth and width variants of the network (other block counts per stage, first-stage width 128 and 32 --
+    the latter takes the gather path for its 32-channel 3x3 convolution) on one image against the oracle."""
+    from paper_2305_14405_b200.harness_cnn import Resnet50Model
+    relu = relu_tables(ctx)
+    x, convs, fc_w, fc_b = nm_inputs_cnn.resnet50_inputs(1, seed=2, random_bn=True, num_classes=64, blocks=blocks,
+                                                         base_width=base)
+    m = Resnet50Model(ctx, 1, convs, fc_w, fc_b, blocks=blocks, base_width=base)
+    logits = m.forward(torch.from_numpy(x).cuda().half())
+    ctx.check_device_status()
+    ref = oracle.cnn.resnet50(x, convs, fc_w, fc_b, relu, blocks=blocks)
+    got = to_np(logits)
+    err = np.abs(got - ref)
+    rms = np.sqrt((ref ** 2).mean())
+    bound = 1e-2 + 1e-2 * np.maximum(np.abs(ref), rms)
+    assert np.all(np.isfinite(got)) and not (err > bound).any(), "%d outside, max err %.4f" % ((err > bound).sum(), err.max())
+
+
+def test_resnet_variant_argument_errors(nm, ctx):
+    from paper_2305_14405_b200.harness_cnn import Resnet50Model
+    cfg = nm.Context.resnet50_cfg(1, nm.F16, blocks=(3, 4, 6, 3), base_width=64)
+    assert ctx.resnet_conv_count(cfg) == 53 and ctx.resnet_conv_count(nm.Context.resnet50_cfg(1, nm.F16)) == 53
+    assert ctx.resnet_conv_count(nm.Context.resnet50_cfg(1, nm.F16, blocks=(3, 4, 23, 3))) == 104
+    for bad in (dict(blocks=(3, 0, 6, 3)), dict(base_width=20), dict(base_width=512), dict(blocks=(1, 1, 1, 99))):
+        c = nm.Context.resnet50_cfg(1, nm.F16, **bad)
+        assert ctx.resnet_conv_count(c) == 0 and ctx.resnet50_workspace_bytes(c) == 0
+
+
 def test_resnet50_host_entry_points_two_streams(nm, ctx):
     """The host-buffer forms: the blocking call equals the device-resident forward bit for bit, and four
     asynchronous calls alternating between two streams (own device buffers and workspaces, different images

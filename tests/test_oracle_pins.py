@@ -757,6 +757,42 @@ def test_resnet50_composition_against_torch():
     assert len(convs) == 53 and sum(c["w"].size for c in convs) + fc_w.size > 23e6   # ResNet-50's ~23.5 M conv weights
 
 
+@pytest.mark.parametrize("blocks,base", [((1, 2, 1, 1), 32), ((2, 1, 1, 2), 16)])
+def test_resnet_variant_composition_against_torch(blocks, base):
+    """The depth / width variants (Section 5 compares ResNet-50 "and its variant models"): the same
+    composition with other block counts per stage and another first-stage width, against
+    torch.nn.functional in fp64; the convolution count and channel widths follow the generator's rule."""
+    import nm_inputs_cnn
+    import oracle.cnn
+    F = torch.nn.functional
+    x, convs, fc_w, fc_b = nm_inputs_cnn.resnet50_inputs(1, seed=5, random_bn=True, image=64, num_classes=8,
+                                                         blocks=blocks, base_width=base)
+    assert len(convs) == 1 + sum(3 * b + 1 for b in blocks)
+    assert convs[0]["w"].shape == (base, 7, 7, 3) and fc_w.shape == (8, 32 * base)
+    assert convs[-1]["w"].shape[0] == 32 * base                      # last block's conv_c: 4 * (base << 3)
+    relu = Table.secant(oracle.RELU, 2, -8.0, 8.0)
+    got = oracle.cnn.resnet50(x, convs, fc_w, fc_b, relu, blocks=blocks)
+
+    def conv(inp, c):
+        _, _, _, s, p = c["spec"]
+        return F.conv2d(inp, torch.from_numpy(c["w"].astype(np.float64)).permute(0, 3, 1, 2),
+                        torch.from_numpy(c["b"].astype(np.float64)), stride=s, padding=p)
+
+    it = iter(convs)
+    y = torch.from_numpy(x.astype(np.float64)).permute(0, 3, 1, 2)
+    y = F.max_pool2d(F.relu(conv(y, next(it))), 3, 2, 1)
+    for nb in blocks:
+        for b in range(nb):
+            ca, cb, cc = next(it), next(it), next(it)
+            t = F.relu(conv(F.relu(conv(y, ca)), cb))
+            sc = conv(y, next(it)) if b == 0 else y
+            y = F.relu(conv(t, cc) + sc)
+    ref = (y.mean(dim=(2, 3)) @ torch.from_numpy(fc_w.astype(np.float64)).T + torch.from_numpy(fc_b.astype(np.float64))).numpy()
+    assert np.allclose(got, ref, rtol=1e-10, atol=1e-9)
+    with pytest.raises((AssertionError, StopIteration)):   # block counts that do not match the convolutions
+        oracle.cnn.resnet50(x, convs, fc_w, fc_b, relu, blocks=(1, 1, 1, 1))
+
+
 # ---------------------------------------------------------------- int8 attention ----------
 
 def _i8_attn_case(B=2, L=24, h=2, d=16, seed=41):
