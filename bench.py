@@ -48,6 +48,8 @@ def parse_args():
     p.add_argument("--layers", type=int, default=0, help="encoder workloads: override the number of layers")
     p.add_argument("--resnet-blocks", default="", help="c5: bottleneck blocks per stage, e.g. 3,4,23,3 (default 3,4,6,3)")
     p.add_argument("--resnet-width", type=int, default=0, help="c5: width of the first stage (default 64)")
+    p.add_argument("--calibrated", action="store_true",
+                   help="encoder workloads: table ranges observed by running the exact model (tests/golden/calibrated_ranges.json)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-rows-leg", action="store_true",
                    help="encoder workloads: skip the row-kernel bandwidth leg on a tensor beyond L2")
@@ -195,6 +197,7 @@ class EncoderWorkload:
         c = self.cfg
         return {"workload": c.name, "layers": c.layers, "batch": c.B, "seq_len": c.L, "hidden": c.H, "heads": c.heads,
                 "ffn": c.F, "pwl_segments": c.segments, "seed": self.args.seed,
+                "table_ranges": "calibrated" if self.args.calibrated else "fixed",
                 "parallelism": "replicas" if world > 1 else "single",
                 "l2": "working set per step (weights %.0f MB + activations %.0f MB) exceeds the 126 MB L2; no flush"
                       % (c.layers * (4 * c.H * c.H + 2 * c.H * c.F) * (1 if c.dtype == "i8" else 2) / 1e6,
@@ -208,7 +211,7 @@ class EncoderWorkload:
         import nm_inputs
         from paper_2305_14405_b200.harness import EncoderModel
         cfg = self.cfg
-        ctx.load_encoder_tables(cfg.segments, cfg.ranges())
+        ctx.load_encoder_tables(cfg.segments, cfg.ranges(self.args.calibrated))
         self.x_np, self.layers_np = nm_inputs.encoder_inputs(cfg, seed=self.args.seed)
         if rank > 0:  # every rank draws its own batch: independent replicas of the same model
             self.x_np, _ = nm_inputs.encoder_inputs(cfg, seed=self.args.seed + rank, layers=0)
@@ -255,7 +258,7 @@ class EncoderWorkload:
     # -- the oracle, as it stands, on whole sampled sequences (sequences are independent) -----------
     def _oracle_tables(self):
         import oracle
-        r = self.cfg.ranges()
+        r = self.cfg.ranges(self.args.calibrated)
         funcs = {"gelu": oracle.GELU, "exp": oracle.EXP, "recip": oracle.RECIP, "rsqrt": oracle.RSQRT}
         return {k: oracle.Table.secant(funcs[k], self.cfg.segments, *r[k]) for k in funcs}
 

@@ -42,9 +42,22 @@ class EncoderConfig:
     def d(self):
         return self.H // self.heads
 
-    def ranges(self):
+    def ranges(self, calibrated=False):
         """[x_min, x_max] of each PWL table: GELU input, exp input (score minus row max),
-        reciprocal input (row sum, at most L), rsqrt input (variance + eps)."""
+        reciprocal input (row sum, at most L), rsqrt input (variance + eps).  The default is fixed per
+        workload; calibrated=True returns the ranges observed by running the exact model on sampled
+        sequences (Section 3.2.1, step 1), as stored by `python -m oracle.calibrate` in
+        tests/golden/calibrated_ranges.json (this module only reads the file)."""
+        if calibrated:
+            import json
+            import os
+            path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "tests", "golden", "calibrated_ranges.json")
+            with open(path) as f:
+                stored = json.load(f)
+            key = self.name.split("_")[0]
+            if key not in stored:
+                raise KeyError("no calibrated ranges stored for %s" % self.name)
+            return {k: tuple(v) for k, v in stored[key]["table"].items()}
         return {"gelu": (-4.0, 4.0), "exp": (-8.0, 0.0), "recip": (self.L / 16.0, float(self.L)),
                 "rsqrt": (0.25, 4.0)}
 

@@ -49,6 +49,29 @@ def test_c2_bert_base_layer_bf16(nm, ctx, algo, random_affine):
     assert_close_bf16(to_np(y), ref, "C2 encoder layer algo %d" % algo)
 
 
+def test_c2_layer_with_calibrated_table_ranges(nm, ctx):
+    """The table ranges observed by running the exact model (Section 3.2.1 step 1; tests/golden/
+    calibrated_ranges.json) instead of the fixed ones: same bound against the oracle with the same tables, and
+    the result is closer to the exact-nonlinearity layer than with the fixed ranges."""
+    cfg = nm_inputs.C2
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=0)
+    m = build(nm, ctx, cfg, layers)
+    exact = {"gelu": oracle.Table.exact(oracle.GELU), "exp": oracle.Table.exact(oracle.EXP),
+             "recip": oracle.Table.exact(oracle.RECIP), "rsqrt": oracle.Table.exact(oracle.RSQRT)}
+    ref_exact = oracle.encoder_layer(x, layers[0], cfg.B, cfg.L, cfg.heads, exact, cfg.eps)
+    dist = {}
+    for mode in (False, True):
+        tabs = load_tables_both(ctx, cfg.segments, cfg.ranges(calibrated=mode))
+        y = m.forward(torch.from_numpy(x).cuda().bfloat16())
+        ctx.check_device_status()
+        ref = oracle.encoder_layer(x, layers[0], cfg.B, cfg.L, cfg.heads, tabs, cfg.eps)
+        assert_close_bf16(to_np(y), ref, "C2 layer, %s ranges" % ("calibrated" if mode else "fixed"))
+        dist[mode] = float(np.sqrt(((ref - ref_exact) ** 2).mean()))
+    print("C2 layer, rms |PWL oracle - exact oracle|: fixed %.3e, calibrated %.3e" % (dist[False], dist[True]))
+    assert dist[True] < dist[False]
+    load_tables_both(ctx, cfg.segments, cfg.ranges())
+
+
 @pytest.mark.parametrize("H,L", [(512, 256), (1024, 128), (1536, 128)])
 def test_width_sweep_layer_bf16(nm, ctx, H, L):
     """Widths of the width/depth sweep (heads of 64, FFN 4H): one layer, two sequences, random biases and

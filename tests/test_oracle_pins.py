@@ -396,6 +396,79 @@ def test_encoder_layer_pwl_approaches_exact_with_more_segments():
     assert errs[2] < 1e-3
 
 
+# ---------------------------------------------------------------- calibrated ranges (Section 3.2.1 step 1)
+
+def test_calibrated_ranges_against_a_torch_run_of_the_exact_layer():
+    """oracle.calibrate records the input range of each nonlinear function while running the exact model;
+    here the same four ranges are taken from an independent fp64 torch run of a small two-layer encoder."""
+    import oracle.calibrate as cal
+    F = torch.nn.functional
+    cfg = nm_inputs.EncoderConfig("t", "f32", B=2, L=16, H=48, heads=4, F=96, layers=2)
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=11, random_affine=True)
+    layers = [{k: v * (5.0 if k.startswith("W") else 1.0) for k, v in w.items()} for w in layers]
+    got = cal.encoder_input_ranges(x, layers, cfg.B, cfg.L, cfg.heads)
+    lo = {k: np.inf for k in got}
+    hi = {k: -np.inf for k in got}
+
+    def see(k, t):
+        lo[k] = min(lo[k], float(t.min()))
+        hi[k] = max(hi[k], float(t.max()))
+
+    y = torch.from_numpy(x.astype(np.float64)).reshape(cfg.B, cfg.L, cfg.H)
+    d = cfg.H // cfg.heads
+    for w in layers:
+        t = {k: torch.from_numpy(np.asarray(v, dtype=np.float64)) for k, v in w.items()}
+        qkv = y @ t["Wqkv"].T + t["bqkv"]
+        q, k, v = (u.reshape(cfg.B, cfg.L, cfg.heads, d).transpose(1, 2) for u in qkv.split(cfg.H, dim=2))
+        s = (q @ k.transpose(2, 3)) / np.sqrt(d)
+        s = s - s.amax(dim=3, keepdim=True)
+        see("exp", s)
+        e = s.exp()
+        see("recip", e.sum(dim=3))
+        a = ((e / e.sum(dim=3, keepdim=True)) @ v).transpose(1, 2).reshape(cfg.B, cfg.L, cfg.H)
+        z1 = y + a @ t["Wo"].T + t["bo"]
+        see("rsqrt", z1.var(dim=2, unbiased=False) + 1e-5)
+        x1 = F.layer_norm(z1, (cfg.H,), t["g1"], t["be1"], 1e-5)
+        pre = x1 @ t["W1"].T + t["b1"]
+        see("gelu", pre)
+        z2 = x1 + F.gelu(pre) @ t["W2"].T + t["b2"]
+        see("rsqrt", z2.var(dim=2, unbiased=False) + 1e-5)
+        y = F.layer_norm(z2, (cfg.H,), t["g2"], t["be2"], 1e-5)
+    for k in got:
+        assert np.isclose(got[k][0], lo[k], rtol=1e-9, atol=1e-12), (k, got[k], lo[k])
+        assert np.isclose(got[k][1], 0.0 if k == "exp" else hi[k], rtol=1e-9, atol=1e-12), (k, got[k], hi[k])
+    assert got["exp"][1] == 0.0 and got["exp"][0] < 0 and 1.0 <= got["recip"][0] <= got["recip"][1] <= cfg.L
+
+
+def test_stored_calibrated_ranges_reproduce_and_tighten_the_tables():
+    """The stored file is what the committed script writes (checked for the small configuration), every table
+    range contains its observed range, and with the calibrated ranges the 64-segment layer is closer to the
+    exact layer than with the fixed ones (the purpose of step 1: segments are not spent outside the data)."""
+    import json
+    import oracle.calibrate as cal
+    with open(cal.GOLDEN) as f:
+        stored = json.load(f)
+    again = cal.calibrate_config("c1")
+    assert again == stored["c1"]
+    for name in ("c1", "c2", "c3"):
+        for k, (a, b) in stored[name]["table"].items():
+            oa, ob = stored[name]["observed"][k]
+            assert a <= oa and ob <= b, (name, k)
+        assert nm_inputs.CONFIGS[name].ranges(calibrated=True) == {k: tuple(v) for k, v in stored[name]["table"].items()}
+    cfg = nm_inputs.C1
+    x, layers = nm_inputs.encoder_inputs(cfg, seed=0)
+    ref = oracle.encoder_layer(x, layers[0], cfg.B, cfg.L, cfg.heads, _exact_tables())
+
+    def err(r):
+        tabs = {"gelu": Table.secant(oracle.GELU, 64, *r["gelu"]), "exp": Table.secant(oracle.EXP, 64, *r["exp"]),
+                "recip": Table.secant(oracle.RECIP, 64, *r["recip"]), "rsqrt": Table.secant(oracle.RSQRT, 64, *r["rsqrt"])}
+        return float(np.abs(oracle.encoder_layer(x, layers[0], cfg.B, cfg.L, cfg.heads, tabs) - ref).max())
+
+    e_fixed, e_cal = err(cfg.ranges()), err(cfg.ranges(calibrated=True))
+    print("C1 layer, 64 segments, max |PWL - exact|: fixed ranges %.3e, calibrated %.3e" % (e_fixed, e_cal))
+    assert e_cal < 0.25 * e_fixed
+
+
 # ---------------------------------------------------------------- int8 -----------
 
 def test_int8_accumulators_and_epilogue():
