@@ -51,6 +51,8 @@ def parse_args():
     p.add_argument("--calibrated", action="store_true",
                    help="encoder workloads: table ranges observed by running the exact model (tests/golden/calibrated_ranges.json)")
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-other-legs", action="store_true",
+                   help="default c3 line: skip the short c4 (int8 encoder) and c5 (CNN) passes reported under other_workloads")
     p.add_argument("--no-rows-leg", action="store_true",
                    help="encoder workloads: skip the row-kernel bandwidth leg on a tensor beyond L2")
     p.add_argument("--repeats", type=int, default=REPEATS, help="how many times the K-step timed region is run")
@@ -622,6 +624,51 @@ def rows_leg(ctx, nm, dev, peaks, peak_kind, hidden=768, rows=1 << 19, iters=20)
     return out
 
 
+def other_workload_leg(name, args, dev, steps=10):
+    """A short device-resident pass of another workload (its own context, tables and buffers; K steps rotating
+    over the streams, CUDA events) so that the default line also carries the int8 encoder's and the CNN's rate."""
+    import copy
+    import torch
+    import paper_2305_14405_b200 as nm
+    a = copy.copy(args)
+    a.workload, a.hidden, a.layers, a.batch, a.calibrated = name, 0, 0, 0, False
+    a.resnet_blocks, a.resnet_width = "", 0
+    wl = make_workload(a)
+    ctx = nm.Context(torch.cuda.current_device())
+    try:
+        wl.setup(ctx, dev, 0)
+        stream = torch.cuda.current_stream()
+        for _ in range(3):
+            wl.step()
+        many = a.streams >= 2 and hasattr(wl, "device_steps")
+        if many:
+            wl.device_steps(4, stream)
+        torch.cuda.synchronize()
+        ctx.check_device_status()
+        ctx.launch_count(reset=True)
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        if many:
+            wl.device_steps(steps, stream)
+        else:
+            for _ in range(steps):
+                wl.step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ctx.check_device_status()
+        ms = e0.elapsed_time(e1) / steps
+        out = {"workload": wl.config(1)["workload"], "metric": wl.metric, "unit": wl.unit, "dtype": wl.dtype,
+               "steps": steps, "streams": a.streams if many else 1, "ms_per_step": ms,
+               "value": wl.units_per_step / (ms * 1e-3), "gpu_launches": ctx.launch_count(),
+               "whole_step_tflops": wl.flops_per_step() / (ms * 1e-3) / 1e12}
+    finally:
+        del wl
+        ctx.close()
+        torch.cuda.empty_cache()
+    return out
+
+
 def main():
     args = parse_args()
     wl = make_workload(args)
@@ -806,6 +853,8 @@ def main():
             line["roofline_rows"] = rows_leg(ctx, nm, dev, peaks, peak_kind)
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = wl.cpu_baseline()
+        if (args.workload == "c3" and not args.no_other_legs and world == 1 and not args.hidden and not args.layers):
+            line["other_workloads"] = [other_workload_leg(n, args, dev) for n in ("c4", "c5")]
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
