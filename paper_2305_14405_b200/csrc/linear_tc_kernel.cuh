@@ -557,9 +557,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
                         if (a.bias) {
 #pragma unroll
-                            for (int i = 0; i < 32; i += 4) {   // zero beyond N
+                            for (int i = 0; i < 32; i += 4) {   // zero beyond N; two columns per packed add
                                 const float4 bs = *reinterpret_cast<const float4*>(my_vec + c * 32 + i);
-                                v[i] += bs.x; v[i + 1] += bs.y; v[i + 2] += bs.z; v[i + 3] += bs.w;
+                                uint64_t s01, s23;
+                                asm("add.rn.f32x2 %0, %1, %2;" : "=l"(s01) : "l"(nm_pack2(v[i], v[i + 1])), "l"(nm_pack2(bs.x, bs.y)));
+                                asm("add.rn.f32x2 %0, %1, %2;" : "=l"(s23) : "l"(nm_pack2(v[i + 2], v[i + 3])), "l"(nm_pack2(bs.z, bs.w)));
+                                nm_unpack2(s01, v[i], v[i + 1]);
+                                nm_unpack2(s23, v[i + 2], v[i + 3]);
                             }
                         }
                     }
@@ -573,8 +577,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                 if (row_ok && col0 + i < a.N) a.idx_dump[row * a.N + col0 + i] = s;
                             }
                         } else {
+                            const uint64_t inv_h2 = nm_pack2(inv_h, inv_h), off2 = nm_pack2(off, off);
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = nm_pwl_fast(rep_lane, v[i], inv_h, off, nm1);
+                            for (int i = 0; i < 32; i += 2) nm_pwl_fast2(rep_lane, v[i], v[i + 1], inv_h2, off2, nm1);
                         }
                     } else if (a.idx_dump) {
 #pragma unroll

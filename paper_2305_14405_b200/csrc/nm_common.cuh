@@ -331,6 +331,40 @@ __device__ __forceinline__ float nm_pwl_fast(uint32_t rep_lane, float x, float i
     return __fmaf_rn(k, x, b);
 }
 
+// Two values at once with the packed fp32 instructions (fma.rn.f32x2, add.rm.f32x2: each half is the same
+// correctly rounded operation as the scalar form, so the results are those of nm_pwl_fast bit for bit).
+__device__ __forceinline__ uint64_t nm_pack2(float a, float b)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void nm_unpack2(uint64_t v, float& a, float& b)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ void nm_pwl_fast2(uint32_t rep_lane, float& x0, float& x1, uint64_t inv_h2, uint64_t off2,
+                                             float nm1)
+{
+    uint64_t u2;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(u2) : "l"(nm_pack2(x0, x1)), "l"(inv_h2), "l"(off2));
+    float u0, u1;
+    nm_unpack2(u2, u0, u1);
+    u0 = fminf(fmaxf(u0, 0.0f), nm1);
+    u1 = fminf(fmaxf(u1, 0.0f), nm1);
+    uint64_t b2;
+    asm("add.rm.f32x2 %0, %1, %2;" : "=l"(b2) : "l"(nm_pack2(u0, u1)), "l"(nm_pack2(12582912.0f, 12582912.0f)));
+    float f0, f1;
+    nm_unpack2(b2, f0, f1);
+    const uint32_t a0 = (__float_as_uint(f0) << 8) + (rep_lane - 0x40000000u);
+    const uint32_t a1 = (__float_as_uint(f1) << 8) + (rep_lane - 0x40000000u);
+    float k0, c0, k1, c1;
+    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(k0), "=f"(c0) : "r"(a0));
+    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(k1), "=f"(c1) : "r"(a1));
+    x0 = __fmaf_rn(k0, x0, c0);
+    x1 = __fmaf_rn(k1, x1, c1);
+}
+
 __device__ __forceinline__ void nm_prefetch_tmap(const CUtensorMap* tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
