@@ -419,6 +419,8 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         // this lane's copy of the replicated table, with the constant of the index trick folded in:
         // (bits << 7) = 0xA0000000 + s*128 (mod 2^32) for bits = 0x4B400000 + s
         const uint32_t rep_lane = nm_smem_u32(rep) + (uint32_t)(lane & 15) * 8u - 0xA0000000u;
+        const uint64_t scale2 = nm_pack2(a.scale, a.scale), inv_h2 = nm_pack2(inv_h, inv_h), off2 = nm_pack2(off, off);
+        const uint64_t magic2 = nm_pack2(12582912.0f, 12582912.0f);
         const uint32_t prow = nm_smem_u32(p_s) + (uint32_t)(g2 * PBUF + row * ROWB);
         const uint32_t p_row = tmem_p + ((uint32_t)(q * 32) << 16);   // this warp's lane quarter of the P columns
         int ok = 1;
@@ -474,6 +476,7 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
             }
             const float neg_ms = -(m * a.scale);
+            const uint64_t neg_ms2 = nm_pack2(neg_ms, neg_ms);
             float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
             // ---- sweep 2: e = PWL_exp(s - m), row sum, P tiles
 #pragma unroll 1
@@ -497,15 +500,33 @@ attention_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         for (int jj = 0; jj < 4; ++jj) {   // 8 keys = one 16-byte chunk of the P row
                             float e[8];
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const float x = __fmaf_rn(__uint_as_float(r[jj * 8 + k]), a.scale, neg_ms);
-                                float u = fmaxf(__fmaf_rn(x, inv_h, off), 0.0f);
-                                if (CLAMP_HI) u = fminf(u, nm1);
+                            for (int k = 0; k < 8; k += 2) {
+                                // two scores at a time on the packed fp32 instructions: each half is the same correctly
+                                // rounded operation as the scalar form
+                                uint64_t x2, u2, b2;
+                                asm("fma.rn.f32x2 %0, %1, %2, %3;"
+                                    : "=l"(x2)
+                                    : "l"(nm_pack2(__uint_as_float(r[jj * 8 + k]), __uint_as_float(r[jj * 8 + k + 1]))), "l"(scale2),
+                                      "l"(neg_ms2));
+                                asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(u2) : "l"(x2), "l"(inv_h2), "l"(off2));
+                                float x0, x1, u0, u1;
+                                nm_unpack2(x2, x0, x1);
+                                nm_unpack2(u2, u0, u1);
+                                u0 = fmaxf(u0, 0.0f);
+                                u1 = fmaxf(u1, 0.0f);
+                                if (CLAMP_HI) {
+                                    u0 = fminf(u0, nm1);
+                                    u1 = fminf(u1, nm1);
+                                }
                                 // floor(u) sits in the low mantissa bits after a round-down add of 1.5 * 2^23
-                                const uint32_t bits = __float_as_uint(__fadd_rd(u, 12582912.0f));
-                                float kk, bb;
-                                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(kk), "=f"(bb) : "r"((bits << 7) + rep_lane));
-                                e[k] = __fmaf_rn(kk, x, bb);
+                                asm("add.rm.f32x2 %0, %1, %2;" : "=l"(b2) : "l"(nm_pack2(u0, u1)), "l"(magic2));
+                                float f0, f1;
+                                nm_unpack2(b2, f0, f1);
+                                float k0, c0, k1, c1;
+                                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(k0), "=f"(c0) : "r"((__float_as_uint(f0) << 7) + rep_lane));
+                                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(k1), "=f"(c1) : "r"((__float_as_uint(f1) << 7) + rep_lane));
+                                e[k] = __fmaf_rn(k0, x0, c0);
+                                e[k + 1] = __fmaf_rn(k1, x1, c1);
                             }
                             sum0 += e[0] + e[4];
                             sum1 += e[1] + e[5];
