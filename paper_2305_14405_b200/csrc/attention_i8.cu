@@ -314,6 +314,8 @@ attention_i8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t rep_lane = nm_smem_u32(rep) + (uint32_t)(lane & 15) * 8u - 0xA0000000u;
         const uint32_t p_row = tmem_p + ((uint32_t)(q * 32) << 16);   // this warp's lane quarter of the P columns
         const float sc = a.sc;
+        const uint64_t sc2 = nm_pack2(sc, sc), inv_h2 = nm_pack2(inv_h, inv_h), off2 = nm_pack2(off, off);
+        const uint64_t magic2 = nm_pack2(12582912.0f, 12582912.0f);
         int ok = 1;
         auto wait_all = [&](uint64_t* bar, uint32_t par) {
             if (!ok) return;
@@ -360,6 +362,7 @@ attention_i8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
             }
             const float neg = -((float)m * sc);
+            const uint64_t neg2 = nm_pack2(neg, neg);
             int isum = 0;
             // ---- sweep 2: exponentials, codes, the integer row sum, P tiles
 #pragma unroll 1
@@ -381,14 +384,31 @@ attention_i8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         for (int w = 0; w < 8; ++w) {
                             float e[4];
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                const float x = __fmaf_rn((float)(int)r[w * 4 + k], sc, neg);
-                                float u = fmaxf(__fmaf_rn(x, inv_h, off), 0.0f);
-                                if (CLAMP_HI) u = fminf(u, nm1);
-                                const uint32_t bits = __float_as_uint(__fadd_rd(u, 12582912.0f));
-                                float kk, bb;
-                                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(kk), "=f"(bb) : "r"((bits << 7) + rep_lane));
-                                e[k] = __fmaf_rn(kk, x, bb);
+                            for (int k = 0; k < 4; k += 2) {
+                                // two scores at a time on the packed fp32 instructions: each half is the same correctly
+                                // rounded operation as the scalar form
+                                uint64_t x2, u2, b2;
+                                asm("fma.rn.f32x2 %0, %1, %2, %3;"
+                                    : "=l"(x2)
+                                    : "l"(nm_pack2((float)(int)r[w * 4 + k], (float)(int)r[w * 4 + k + 1])), "l"(sc2), "l"(neg2));
+                                asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(u2) : "l"(x2), "l"(inv_h2), "l"(off2));
+                                float x0, x1, u0, u1;
+                                nm_unpack2(x2, x0, x1);
+                                nm_unpack2(u2, u0, u1);
+                                u0 = fmaxf(u0, 0.0f);
+                                u1 = fmaxf(u1, 0.0f);
+                                if (CLAMP_HI) {
+                                    u0 = fminf(u0, nm1);
+                                    u1 = fminf(u1, nm1);
+                                }
+                                asm("add.rm.f32x2 %0, %1, %2;" : "=l"(b2) : "l"(nm_pack2(u0, u1)), "l"(magic2));
+                                float f0, f1;
+                                nm_unpack2(b2, f0, f1);
+                                float k0, c0, k1, c1;
+                                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(k0), "=f"(c0) : "r"((__float_as_uint(f0) << 7) + rep_lane));
+                                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(k1), "=f"(c1) : "r"((__float_as_uint(f1) << 7) + rep_lane));
+                                e[k] = __fmaf_rn(k0, x0, c0);
+                                e[k + 1] = __fmaf_rn(k1, x1, c1);
                             }
                             pk[w] = nm_quant_i8x4(e[0], e[1], e[2], e[3], 127.0f);
                             isum = __dp4a((int)pk[w], 0x01010101, isum);
