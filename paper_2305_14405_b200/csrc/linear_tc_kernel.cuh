@@ -547,10 +547,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             if (a.acc_dump && row_ok && col0 + i < a.N)
                                 *reinterpret_cast<int4*>(a.acc_dump + row * a.N + col0 + i) =
                                     make_int4((int)r[i], (int)r[i + 1], (int)r[i + 2], (int)r[i + 3]);
-                            v[i] = __fmaf_rn((float)(int)r[i], ws.x, bs.x);
-                            v[i + 1] = __fmaf_rn((float)(int)r[i + 1], ws.y, bs.y);
-                            v[i + 2] = __fmaf_rn((float)(int)r[i + 2], ws.z, bs.z);
-                            v[i + 3] = __fmaf_rn((float)(int)r[i + 3], ws.w, bs.w);
+                            uint64_t d01, d23;   // fma((float)acc, scale, bias), two columns per packed instruction
+                            asm("fma.rn.f32x2 %0, %1, %2, %3;"
+                                : "=l"(d01)
+                                : "l"(nm_pack2((float)(int)r[i], (float)(int)r[i + 1])), "l"(nm_pack2(ws.x, ws.y)), "l"(nm_pack2(bs.x, bs.y)));
+                            asm("fma.rn.f32x2 %0, %1, %2, %3;"
+                                : "=l"(d23)
+                                : "l"(nm_pack2((float)(int)r[i + 2], (float)(int)r[i + 3])), "l"(nm_pack2(ws.z, ws.w)),
+                                  "l"(nm_pack2(bs.z, bs.w)));
+                            nm_unpack2(d01, v[i], v[i + 1]);
+                            nm_unpack2(d23, v[i + 2], v[i + 3]);
                         }
                     } else {
 #pragma unroll
