@@ -850,11 +850,20 @@ def main():
             "whole_step_tflops": whole,
         }
         if isinstance(wl, EncoderWorkload) and not args.no_rows_leg and world == 1:
-            line["roofline_rows"] = rows_leg(ctx, nm, dev, peaks, peak_kind)
+            try:
+                line["roofline_rows"] = rows_leg(ctx, nm, dev, peaks, peak_kind)
+            except Exception as e:   # noqa: BLE001 - reported, not hidden
+                line["roofline_rows"] = {"error": "%s: %s" % (type(e).__name__, e)}
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = wl.cpu_baseline()
         if (args.workload == "c3" and not args.no_other_legs and world == 1 and not args.hidden and not args.layers):
-            line["other_workloads"] = [other_workload_leg(n, args, dev) for n in ("c4", "c5")]
+            legs = []
+            for n in ("c4", "c5"):   # a failure here must not cost the main line
+                try:
+                    legs.append(other_workload_leg(n, args, dev))
+                except Exception as e:   # noqa: BLE001 - reported, not hidden
+                    legs.append({"workload": n, "error": "%s: %s" % (type(e).__name__, e)})
+            line["other_workloads"] = legs
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
